@@ -1,0 +1,346 @@
+/*
+ * CPU oracle for k-MIP self-attention  --  TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, fp64 restatement of what the method computes, used only by the
+ * tests, the smoke check and the benchmark's cpu_baseline leg.  It shares no code
+ * with the CUDA library and must never be called from the product path.
+ *
+ * What it follows:
+ *   forward   Eq. 1 and Algorithm 1 lines 2-6 of the paper: for every head h and
+ *             query node i, all inner products q_i . k_j over the nodes j of i's own
+ *             graph (self included, Eq. 1 has no diagonal mask); keep the k largest
+ *             (T_k: everything else is -inf); softmax of (kept score / sqrt(d_K));
+ *             weighted sum of the kept V rows.  The 1/sqrt(d_K) factor sits outside
+ *             T_k in Eq. 1 and in line 5 of Algorithm 1, so selection and the stored
+ *             E_topk use the raw inner product.
+ *   backward  chain rule through lines 4-6 of Algorithm 1 with the index set held
+ *             constant (Sec. 3.1: the top-k indices are reused in the sparse backward;
+ *             App. E: I_argtopk and E_topk need no recomputation).
+ *
+ * Readings where the paper is silent: ties are broken by the lower key index; the k
+ * results are ordered by (score descending, index ascending); indices are global row
+ * numbers of the concatenated batch; a graph with fewer than k nodes keeps all of them
+ * and pads the remaining slots with index -1 / score -inf / weight 0; graphs of a
+ * batch are separated by CSR offsets; NaN scores count as -inf.
+ *
+ * Inputs are float arrays (bf16- or fp32-valued); every product and sum is fp64.
+ * Layout: Q, K, V, dOut, out, dQ, dK, dV : [N, H, d] row-major.
+ *
+ * Parity pins (tests/test_oracle_pins.py): k = n equals dense softmax attention
+ * (library routine), k = 1 equals arg-max retrieval, exhaustive subset enumeration on
+ * tiny cases, hand-derived closed-form fixtures, constant-V and identical-K cases,
+ * permutation equivariance, CSR confinement, finite differences and autograd for the
+ * backward.  No function here is unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define KMIP_ORACLE_OK 0
+#define KMIP_ORACLE_BAD_ARG 1
+#define KMIP_ORACLE_NOMEM 2
+
+int kmip_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* q . k over d entries in fp64, index order (Algorithm 1 line 2, one entry of S). */
+static double inner(const float *q, const float *kk, int d)
+{
+    double s = 0.0;
+    for (int c = 0; c < d; ++c)
+        s += (double)q[c] * (double)kk[c];
+    return s;
+}
+
+/* Node range [lo, hi) of the graph that holds row i. */
+static int graph_range(const int32_t *offs, int32_t G, int64_t N, int64_t i, int64_t *lo, int64_t *hi)
+{
+    if (offs == NULL) {
+        *lo = 0;
+        *hi = N;
+        return 1;
+    }
+    for (int32_t g = 0; g < G; ++g)
+        if ((int64_t)offs[g] <= i && i < (int64_t)offs[g + 1]) {
+            *lo = offs[g];
+            *hi = offs[g + 1];
+            return 1;
+        }
+    return 0;
+}
+
+static int offsets_ok(const int32_t *offs, int32_t G, int64_t N)
+{
+    if (offs == NULL)
+        return 1;
+    if (G < 0 || offs[0] != 0 || (int64_t)offs[G] != N)
+        return 0;
+    for (int32_t g = 0; g < G; ++g)
+        if (offs[g] > offs[g + 1])
+            return 0;
+    return 1;
+}
+
+/*
+ * Row-wise top-k (Algorithm 1 line 3) as a partial insertion sort: walk the keys in
+ * index order and keep a list of at most `keep` entries sorted by (score desc, index
+ * asc).  A new score goes after every entry whose score is >= its own, so among equal
+ * scores the lower index stays in front.
+ */
+static void topk_insert(double *ls, int64_t *li, int *len, int keep, double s, int64_t j)
+{
+    int p = *len;
+    while (p > 0 && ls[p - 1] < s)
+        --p;
+    if (p >= keep)
+        return;
+    int last = (*len < keep) ? *len : keep - 1;
+    for (int t = last; t > p; --t) {
+        ls[t] = ls[t - 1];
+        li[t] = li[t - 1];
+    }
+    ls[p] = s;
+    li[p] = j;
+    if (*len < keep)
+        ++*len;
+}
+
+/* softmax over `n` kept scores scaled by 1/sqrt(d) (Algorithm 1 line 5). */
+static void softmax_scaled(const double *s, int n, double scale, double *p)
+{
+    double m = -INFINITY, z = 0.0;
+    for (int t = 0; t < n; ++t)
+        if (s[t] > m)
+            m = s[t];
+    for (int t = 0; t < n; ++t) {
+        p[t] = exp(scale * (s[t] - m));
+        z += p[t];
+    }
+    for (int t = 0; t < n; ++t)
+        p[t] /= z;
+}
+
+/*
+ * Forward for the query rows listed in `rows` (rows == NULL: all N rows, n_rows = N).
+ * Outputs are indexed by position in `rows`:
+ *   out [n_rows, H, d] fp64, topk_idx [n_rows, H, k] int32, topk_score [n_rows, H, k] fp64,
+ *   kth_gap [n_rows, H] fp64 (optional): score of the k-th kept key minus the best
+ *   score left out (+inf when nothing is left out) -- how far the selection is from a tie.
+ */
+int kmip_oracle_forward_rows(const float *Q, const float *K, const float *V,
+                             const int32_t *graph_offsets, int32_t G, int64_t N,
+                             int32_t H, int32_t d, int32_t k,
+                             const int64_t *rows, int64_t n_rows,
+                             double *out, int32_t *topk_idx, double *topk_score, double *kth_gap)
+{
+    if (!Q || !K || !V || !out || !topk_idx || !topk_score || N < 0 || H < 1 || d < 1 || k < 1)
+        return KMIP_ORACLE_BAD_ARG;
+    if (!offsets_ok(graph_offsets, G, N))
+        return KMIP_ORACLE_BAD_ARG;
+    if (rows == NULL)
+        n_rows = N;
+    const double scale = 1.0 / sqrt((double)d);
+    const int64_t HD = (int64_t)H * d;
+    int failed = 0;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const int64_t i = rows ? rows[r] : r;
+        int64_t lo, hi;
+        double *ls = (double *)malloc(sizeof(double) * (size_t)(k + 1));
+        int64_t *li = (int64_t *)malloc(sizeof(int64_t) * (size_t)(k + 1));
+        double *p = (double *)malloc(sizeof(double) * (size_t)k);
+        if (!ls || !li || !p || i < 0 || i >= N || !graph_range(graph_offsets, G, N, i, &lo, &hi)) {
+            failed = 1;
+        } else {
+            for (int32_t h = 0; h < H; ++h) {
+                const float *q = Q + i * HD + (int64_t)h * d;
+                int len = 0;
+                /* all scores of the row, reduced on the fly to the best k+1 */
+                for (int64_t j = lo; j < hi; ++j) {
+                    double s = inner(q, K + j * HD + (int64_t)h * d, d);
+                    if (isnan(s))
+                        s = -INFINITY;
+                    topk_insert(ls, li, &len, k + 1, s, j);
+                }
+                const int keff = len < k ? len : k;
+                int32_t *oi = topk_idx + (r * H + h) * (int64_t)k;
+                double *os = topk_score + (r * H + h) * (int64_t)k;
+                for (int t = 0; t < k; ++t) {
+                    oi[t] = t < keff ? (int32_t)li[t] : -1;
+                    os[t] = t < keff ? ls[t] : -INFINITY;
+                }
+                if (kth_gap)
+                    kth_gap[r * H + h] = (len > k) ? ls[k - 1] - ls[k] : INFINITY;
+                double *o = out + (r * H + h) * (int64_t)d;
+                for (int c = 0; c < d; ++c)
+                    o[c] = 0.0;
+                if (keff > 0) {
+                    softmax_scaled(ls, keff, scale, p);
+                    /* gather the kept V rows and sum them with their weights (lines 4 and 6) */
+                    for (int t = 0; t < keff; ++t) {
+                        const float *v = V + li[t] * HD + (int64_t)h * d;
+                        for (int c = 0; c < d; ++c)
+                            o[c] += p[t] * (double)v[c];
+                    }
+                }
+            }
+        }
+        free(ls);
+        free(li);
+        free(p);
+    }
+    return failed ? KMIP_ORACLE_BAD_ARG : KMIP_ORACLE_OK;
+}
+
+/*
+ * Lines 4-6 of Algorithm 1 for an index set supplied by the caller (any order, -1 = empty
+ * slot); the scores of the listed keys are recomputed in fp64.
+ *   idx [n_rows, H, k], out [n_rows, H, d], score_out [n_rows, H, k] (optional).
+ */
+int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V,
+                                  int64_t N, int32_t H, int32_t d, int32_t k,
+                                  const int64_t *rows, int64_t n_rows, const int32_t *idx,
+                                  double *out, double *score_out)
+{
+    if (!Q || !K || !V || !idx || !out || N < 0 || H < 1 || d < 1 || k < 1)
+        return KMIP_ORACLE_BAD_ARG;
+    if (rows == NULL)
+        n_rows = N;
+    const double scale = 1.0 / sqrt((double)d);
+    const int64_t HD = (int64_t)H * d;
+    int failed = 0;
+
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const int64_t i = rows ? rows[r] : r;
+        double *s = (double *)malloc(sizeof(double) * (size_t)k);
+        double *p = (double *)malloc(sizeof(double) * (size_t)k);
+        int64_t *jj = (int64_t *)malloc(sizeof(int64_t) * (size_t)k);
+        if (!s || !p || !jj || i < 0 || i >= N) {
+            failed = 1;
+        } else {
+            for (int32_t h = 0; h < H; ++h) {
+                const int32_t *ii = idx + (r * H + h) * (int64_t)k;
+                const float *q = Q + i * HD + (int64_t)h * d;
+                int n = 0;
+                for (int t = 0; t < k; ++t) {
+                    if (score_out)
+                        score_out[(r * H + h) * (int64_t)k + t] = -INFINITY;
+                    if (ii[t] < 0)
+                        continue;
+                    if (ii[t] >= N) {
+                        failed = 1;
+                        continue;
+                    }
+                    jj[n] = ii[t];
+                    s[n] = inner(q, K + jj[n] * HD + (int64_t)h * d, d);
+                    if (score_out)
+                        score_out[(r * H + h) * (int64_t)k + t] = s[n];
+                    ++n;
+                }
+                double *o = out + (r * H + h) * (int64_t)d;
+                for (int c = 0; c < d; ++c)
+                    o[c] = 0.0;
+                if (n > 0) {
+                    softmax_scaled(s, n, scale, p);
+                    for (int t = 0; t < n; ++t) {
+                        const float *v = V + jj[t] * HD + (int64_t)h * d;
+                        for (int c = 0; c < d; ++c)
+                            o[c] += p[t] * (double)v[c];
+                    }
+                }
+            }
+        }
+        free(s);
+        free(p);
+        free(jj);
+    }
+    return failed ? KMIP_ORACLE_BAD_ARG : KMIP_ORACLE_OK;
+}
+
+/*
+ * Backward through lines 4-6 of Algorithm 1 with the selection held constant.
+ * With s_t = q_i . k_{j_t}, p = softmax(s / sqrt(d)), o_i = sum_t p_t v_{j_t} and upstream g_i:
+ *   dP_t = g_i . v_{j_t}          D = sum_t p_t dP_t        dS_t = p_t (dP_t - D) / sqrt(d)
+ *   dQ_i += dS_t k_{j_t}          dK_{j_t} += dS_t q_i      dV_{j_t} += p_t g_i
+ * idx [N, H, k] (-1 = empty slot).  dQ, dK, dV [N, H, d] fp64, overwritten.
+ * Heads touch disjoint columns, so the loop over heads is the parallel one.
+ */
+int kmip_oracle_backward(const float *Q, const float *K, const float *V, const float *dOut,
+                         const int32_t *idx, int64_t N, int32_t H, int32_t d, int32_t k,
+                         double *dQ, double *dK, double *dV)
+{
+    if (!Q || !K || !V || !dOut || !idx || !dQ || !dK || !dV || N < 0 || H < 1 || d < 1 || k < 1)
+        return KMIP_ORACLE_BAD_ARG;
+    const double scale = 1.0 / sqrt((double)d);
+    const int64_t HD = (int64_t)H * d;
+    memset(dQ, 0, sizeof(double) * (size_t)(N * HD));
+    memset(dK, 0, sizeof(double) * (size_t)(N * HD));
+    memset(dV, 0, sizeof(double) * (size_t)(N * HD));
+    int failed = 0;
+
+#pragma omp parallel for schedule(static, 1)
+    for (int32_t h = 0; h < H; ++h) {
+        double *s = (double *)malloc(sizeof(double) * (size_t)k);
+        double *p = (double *)malloc(sizeof(double) * (size_t)k);
+        double *dP = (double *)malloc(sizeof(double) * (size_t)k);
+        int64_t *jj = (int64_t *)malloc(sizeof(int64_t) * (size_t)k);
+        if (!s || !p || !dP || !jj) {
+            failed = 1;
+        } else {
+            for (int64_t i = 0; i < N; ++i) {
+                const int32_t *ii = idx + (i * H + h) * (int64_t)k;
+                const float *q = Q + i * HD + (int64_t)h * d;
+                const float *g = dOut + i * HD + (int64_t)h * d;
+                int n = 0;
+                for (int t = 0; t < k; ++t) {
+                    if (ii[t] < 0)
+                        continue;
+                    if (ii[t] >= N) {
+                        failed = 1;
+                        continue;
+                    }
+                    jj[n] = ii[t];
+                    s[n] = inner(q, K + jj[n] * HD + (int64_t)h * d, d);
+                    ++n;
+                }
+                if (n == 0)
+                    continue;
+                softmax_scaled(s, n, scale, p);
+                double D = 0.0;
+                for (int t = 0; t < n; ++t) {
+                    dP[t] = inner(g, V + jj[t] * HD + (int64_t)h * d, d);
+                    D += p[t] * dP[t];
+                }
+                for (int t = 0; t < n; ++t) {
+                    const double dS = scale * p[t] * (dP[t] - D);
+                    const float *kr = K + jj[t] * HD + (int64_t)h * d;
+                    double *dq = dQ + i * HD + (int64_t)h * d;
+                    double *dk = dK + jj[t] * HD + (int64_t)h * d;
+                    double *dv = dV + jj[t] * HD + (int64_t)h * d;
+                    for (int c = 0; c < d; ++c) {
+                        dq[c] += dS * (double)kr[c];
+                        dk[c] += dS * (double)q[c];
+                        dv[c] += p[t] * (double)g[c];
+                    }
+                }
+            }
+        }
+        free(s);
+        free(p);
+        free(dP);
+        free(jj);
+    }
+    return failed ? KMIP_ORACLE_BAD_ARG : KMIP_ORACLE_OK;
+}

@@ -1,0 +1,116 @@
+"""ctypes front end of the fp64 CPU oracle (TEST INFRASTRUCTURE, NOT THE PRODUCT).
+
+Only the tests, the smoke check and the benchmark's cpu_baseline / reference leg may
+import this module.  It compiles `kmip_oracle.c` with gcc on first use (or when the
+source is newer than the shared object) and marshals numpy arrays; all arithmetic is
+in the C file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kmip_oracle.c")
+_LIB = os.path.join(_HERE, "libkmip_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc -O2 -fopenmp; returns the path of the shared object."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared",
+                               "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        P = ctypes.c_void_p
+        i32, i64 = ctypes.c_int32, ctypes.c_int64
+        lib.kmip_oracle_threads.restype = ctypes.c_int
+        lib.kmip_oracle_forward_rows.restype = ctypes.c_int
+        lib.kmip_oracle_forward_rows.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, P, i64, P, P, P, P]
+        lib.kmip_oracle_forward_given_idx.restype = ctypes.c_int
+        lib.kmip_oracle_forward_given_idx.argtypes = [P, P, P, i64, i32, i32, i32, P, i64, P, P, P]
+        lib.kmip_oracle_backward.restype = ctypes.c_int
+        lib.kmip_oracle_backward.argtypes = [P, P, P, P, P, i64, i32, i32, i32, P, P, P]
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    return int(_load().kmip_oracle_threads())
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    assert a.ndim == 3
+    return a
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def forward(Q, K, V, graph_offsets, k, rows=None):
+    """Oracle forward.  Returns dict(out, idx, score, gap); arrays are indexed by position
+    in `rows` (all rows when rows is None)."""
+    Q, K, V = _f32(Q), _f32(K), _f32(V)
+    N, H, d = Q.shape
+    offs = None if graph_offsets is None else np.ascontiguousarray(graph_offsets, dtype=np.int32)
+    G = 1 if offs is None else len(offs) - 1
+    rws = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = N if rws is None else len(rws)
+    out = np.zeros((n, H, d), dtype=np.float64)
+    idx = np.full((n, H, k), -1, dtype=np.int32)
+    score = np.full((n, H, k), -np.inf, dtype=np.float64)
+    gap = np.full((n, H), np.inf, dtype=np.float64)
+    rc = _load().kmip_oracle_forward_rows(_ptr(Q), _ptr(K), _ptr(V), _ptr(offs), G, N, H, d, k,
+                                          _ptr(rws), n, _ptr(out), _ptr(idx), _ptr(score), _ptr(gap))
+    if rc != 0:
+        raise ValueError(f"kmip_oracle_forward_rows failed with status {rc}")
+    return {"out": out, "idx": idx, "score": score, "gap": gap}
+
+
+def forward_given_idx(Q, K, V, idx, rows=None):
+    """Softmax-weighted sum over a caller-supplied index set; returns (out, score)."""
+    Q, K, V = _f32(Q), _f32(K), _f32(V)
+    N, H, d = Q.shape
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    rws = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = N if rws is None else len(rws)
+    assert idx.shape[0] == n and idx.shape[1] == H
+    k = idx.shape[2]
+    out = np.zeros((n, H, d), dtype=np.float64)
+    score = np.zeros((n, H, k), dtype=np.float64)
+    rc = _load().kmip_oracle_forward_given_idx(_ptr(Q), _ptr(K), _ptr(V), N, H, d, k,
+                                               _ptr(rws), n, _ptr(idx), _ptr(out), _ptr(score))
+    if rc != 0:
+        raise ValueError(f"kmip_oracle_forward_given_idx failed with status {rc}")
+    return out, score
+
+
+def backward(Q, K, V, dOut, idx):
+    """Sparse backward with the selection held constant; returns (dQ, dK, dV) in fp64."""
+    Q, K, V, dOut = _f32(Q), _f32(K), _f32(V), _f32(dOut)
+    N, H, d = Q.shape
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    assert idx.shape[:2] == (N, H)
+    k = idx.shape[2]
+    dQ = np.empty((N, H, d), dtype=np.float64)
+    dK = np.empty((N, H, d), dtype=np.float64)
+    dV = np.empty((N, H, d), dtype=np.float64)
+    rc = _load().kmip_oracle_backward(_ptr(Q), _ptr(K), _ptr(V), _ptr(dOut), _ptr(idx), N, H, d, k,
+                                      _ptr(dQ), _ptr(dK), _ptr(dV))
+    if rc != 0:
+        raise ValueError(f"kmip_oracle_backward failed with status {rc}")
+    return dQ, dK, dV
