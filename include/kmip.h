@@ -1,0 +1,128 @@
+/*
+ * kmip.h -- C ABI of the B200 (sm_100a) k-Maximum-Inner-Product self-attention library.
+ *
+ * The library computes the hot path of multi-head k-MIP self-attention (Eq. 1-2 and
+ * Algorithm 1, lines 2-6, of "k-Maximum Inner Product Attention for Graph Transformers")
+ * and its sparse backward pass (Sec. 3.1: the top-k indices are reused, the search is
+ * not repeated), for a batch of graphs stored back to back and delimited by CSR offsets.
+ *
+ * Conventions shared by every call
+ *   N        total number of nodes of the batch (all graphs concatenated), 0 <= N < 2^31
+ *   G        number of graphs; graph g owns rows graph_offsets[g] .. graph_offsets[g+1]-1
+ *   H, d, k  heads, per-head width (d_K = d_V = d), keys kept per query
+ *   layouts  Q, K, V, out, d_out, dQ, dK, dV : [N, H, d] row-major (a node's H*d values are
+ *            contiguous, head h at columns h*d .. h*d+d-1);
+ *            topk_idx : int32 [N, H, k];  topk_score : float [N, H, k];
+ *            graph_offsets : int32 [G+1], offsets[0] = 0, non-decreasing, offsets[G] = N.
+ *   memory   every pointer is DEVICE memory owned by the caller, 16-byte aligned, and stays
+ *            valid until the work enqueued on `stream` has finished.  The library allocates
+ *            no device memory and keeps no state between calls; `workspace` is caller-owned
+ *            scratch whose contents are undefined between calls.  Its first 256 bytes are
+ *            a status block that kmip_last_status reads.
+ *   async    calls validate their arguments on the host, enqueue kernels on `stream`
+ *            (a cudaStream_t passed as void*, NULL = default stream) and return without
+ *            synchronising.  KMIP_OK means "enqueued".  Problems only the device can see
+ *            (malformed offsets, an expired bounded wait) are recorded in the status block.
+ *   errors   nothing is enqueued when a call returns a status other than KMIP_OK.
+ */
+#ifndef KMIP_H_
+#define KMIP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KMIP_OK = 0,
+    KMIP_ERR_INVALID_ARG = 1,  /* null or misaligned pointer, negative size, k < 1, H < 1, N*H*k >= 2^31 */
+    KMIP_ERR_UNSUPPORTED = 2,  /* d not in {16, 32, 64, 128}, k > 128, unknown mode */
+    KMIP_ERR_WORKSPACE = 3,    /* workspace smaller than kmip_attn_workspace_bytes reports */
+    KMIP_ERR_CUDA = 4,         /* a CUDA runtime call or a kernel launch failed */
+    KMIP_ERR_TIMEOUT = 5,      /* device side: a bounded wait inside a kernel ran out */
+    KMIP_ERR_BAD_OFFSETS = 6   /* device side: graph_offsets is not a valid CSR row-pointer array */
+} kmip_status_t;
+
+typedef enum {
+    /* Q, K, V, out, d_out, dQ, dK, dV hold bf16.  Scores are a dense bf16 contraction with fp32
+       accumulation on the tcgen05 tensor cores; softmax, sums and gradients accumulate in fp32. */
+    KMIP_BF16_TC = 0,
+    /* All of them hold fp32.  Scores are fp32 fused multiply-adds in index order c = 0..d-1. */
+    KMIP_FP32_EXACT = 1
+} kmip_mode_t;
+
+#define KMIP_PASS_FORWARD 0
+#define KMIP_PASS_BACKWARD 1
+
+/*
+ * Scratch size in bytes that kmip_attn_forward (pass = 0) or kmip_attn_backward (pass = 1)
+ * needs for this problem size.  Linear in N*H*(k + 1): the N x N score matrix of Algorithm 1
+ * line 2 is never stored (Sec. 3.1, App. F).  Host only, no CUDA call.
+ */
+int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k,
+                              int mode, int pass, size_t *bytes);
+
+/*
+ * Forward pass, Eq. 1 and Algorithm 1 lines 2-6, for every head h and every query node i:
+ *   s_ij       = q_i^h . k_j^h   for all nodes j of i's own graph (self included)
+ *   topk       : the k largest s_ij; ties go to the lower j; listed by (score desc, j asc)
+ *   topk_idx   = their global row numbers j        (I_argtopk of Algorithm 1 line 3)
+ *   topk_score = their raw inner products s_ij     (E_topk; the 1/sqrt(d) factor is not applied here)
+ *   out[i,h,:] = sum_t softmax_t(topk_score / sqrt(d)) * V[topk_idx_t, h, :]   (lines 4-6)
+ * A graph with n < k nodes keeps all n and pads: topk_idx = -1, topk_score = -inf, weight 0.
+ * graph_offsets may be NULL, meaning one graph [0, N) (G is then ignored).
+ * N = 0 returns KMIP_OK and enqueues nothing.
+ * Inputs: Q, K, V, graph_offsets.  Outputs (fully overwritten): out, topk_idx, topk_score.
+ * In KMIP_BF16_TC mode the selection uses tensor-core scores, so a key whose exact score
+ * differs from the k-th best by less than the fp32 accumulation error may swap with it.
+ */
+int kmip_attn_forward(const void *Q, const void *K, const void *V,
+                      const int32_t *graph_offsets, int32_t G, int64_t N,
+                      int32_t H, int32_t d, int32_t k, int mode,
+                      void *out, int32_t *topk_idx, float *topk_score,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Backward pass through Algorithm 1 lines 4-6 with the selection held constant (Sec. 3.1,
+ * App. E: I_argtopk and E_topk are reused).  With p = softmax(topk_score / sqrt(d)) and
+ * upstream gradient g = d_out:
+ *   dP_t = g_i . v_{j_t}     D = sum_t p_t dP_t     dS_t = p_t (dP_t - D) / sqrt(d)
+ *   dQ[i,h,:] = sum_t dS_t K[j_t,h,:]
+ *   dK[m,h,:] = sum over (i,t) with j_t = m of dS_t Q[i,h,:]
+ *   dV[m,h,:] = sum over (i,t) with j_t = m of p_t g[i,h,:]
+ * Slots with topk_idx < 0 are ignored; keys nobody selected get zero gradient.
+ * Inputs: Q, K, V, d_out, topk_idx, topk_score as written by kmip_attn_forward on the same
+ * Q, K; `out` is accepted for symmetry with autograd interfaces and may be NULL.
+ * Outputs (fully overwritten): dQ, dK, dV.  graph_offsets and G are not needed by the
+ * arithmetic (indices are global) and may be NULL / 0.
+ * dK and dV are sums over an unordered list of hits: results are reproducible to fp32
+ * rounding of the summation order, not bit for bit.
+ */
+int kmip_attn_backward(const void *Q, const void *K, const void *V,
+                       const int32_t *graph_offsets, int32_t G, int64_t N,
+                       int32_t H, int32_t d, int32_t k, int mode,
+                       const void *out, const void *d_out,
+                       const int32_t *topk_idx, const float *topk_score,
+                       void *dQ, void *dK, void *dV,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Synchronises `stream`, then copies the device status word of the last call that used
+ * `workspace` into *device_status (KMIP_OK, KMIP_ERR_TIMEOUT or KMIP_ERR_BAD_OFFSETS).
+ * Returns KMIP_ERR_CUDA if the synchronisation or the copy fails.  For tests and debugging;
+ * not needed on the hot path.
+ */
+int kmip_last_status(const void *workspace, void *stream, int *device_status);
+
+/* Static, NUL-terminated description of a status code. */
+const char *kmip_status_string(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int kmip_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KMIP_H_ */

@@ -1,0 +1,187 @@
+"""Thin Python binding of the C-ABI library `libkmip.so` (argument marshalling only).
+
+Function names follow `include/kmip.h`.  Tensors are torch CUDA tensors used purely as
+device buffers; every step of the computation runs inside the library's CUDA kernels.
+There is no CPU or PyTorch fallback: if the shared library is missing the import fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+KMIP_OK = 0
+KMIP_ERR_INVALID_ARG = 1
+KMIP_ERR_UNSUPPORTED = 2
+KMIP_ERR_WORKSPACE = 3
+KMIP_ERR_CUDA = 4
+KMIP_ERR_TIMEOUT = 5
+KMIP_ERR_BAD_OFFSETS = 6
+KMIP_BF16_TC = 0
+KMIP_FP32_EXACT = 1
+PASS_FORWARD = 0
+PASS_BACKWARD = 1
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libkmip.so")
+_lib = None
+
+
+class KmipError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2604_03815_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        P, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        L.kmip_version.restype = ctypes.c_int
+        L.kmip_status_string.restype = ctypes.c_char_p
+        L.kmip_status_string.argtypes = [ctypes.c_int]
+        L.kmip_attn_workspace_bytes.restype = ctypes.c_int
+        L.kmip_attn_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, ctypes.c_int, ctypes.c_int,
+                                                ctypes.POINTER(sz)]
+        L.kmip_attn_forward.restype = ctypes.c_int
+        L.kmip_attn_forward.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, P, P, P, P, sz, P]
+        L.kmip_attn_backward.restype = ctypes.c_int
+        L.kmip_attn_backward.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, P, P, P, P,
+                                         P, P, P, P, sz, P]
+        L.kmip_last_status.restype = ctypes.c_int
+        L.kmip_last_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_int)]
+        L.kmip_debug_tc_scores.restype = ctypes.c_int
+        L.kmip_debug_tc_scores.argtypes = [P, P, i64, i32, i32, P, P, sz, P]
+        _lib = L
+    return _lib
+
+
+def kmip_version() -> int:
+    return int(lib().kmip_version())
+
+
+def status_string(status: int) -> str:
+    return lib().kmip_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def kmip_attn_workspace_bytes(N, G, H, d, k, mode, pass_) -> int:
+    out = ctypes.c_size_t(0)
+    rc = lib().kmip_attn_workspace_bytes(N, G, H, d, k, mode, pass_, ctypes.byref(out))
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_attn_workspace_bytes")
+    return int(out.value)
+
+
+def kmip_attn_forward(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score, workspace, stream=None) -> int:
+    """Enqueue the forward pass; returns the library's status code (no exception, no sync)."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(lib().kmip_attn_forward(_ptr(Q), _ptr(K), _ptr(V), _ptr(graph_offsets), G, N, H, d, k, mode,
+                                       _ptr(out), _ptr(topk_idx), _ptr(topk_score), _ptr(workspace),
+                                       0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                       _stream(stream)))
+
+
+def kmip_attn_backward(Q, K, V, graph_offsets, k, mode, out, d_out, topk_idx, topk_score, dQ, dK, dV,
+                       workspace, stream=None) -> int:
+    """Enqueue the backward pass; returns the library's status code (no exception, no sync)."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(lib().kmip_attn_backward(_ptr(Q), _ptr(K), _ptr(V), _ptr(graph_offsets), G, N, H, d, k, mode,
+                                        _ptr(out), _ptr(d_out), _ptr(topk_idx), _ptr(topk_score),
+                                        _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(workspace),
+                                        0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                        _stream(stream)))
+
+
+def kmip_last_status(workspace, stream=None) -> int:
+    """Synchronise the stream and return the device-side status recorded in the workspace."""
+    st = ctypes.c_int(0)
+    rc = lib().kmip_last_status(_ptr(workspace), _stream(stream), ctypes.byref(st))
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_last_status")
+    return int(st.value)
+
+
+def kmip_debug_tc_scores(Q, K, scores, workspace, stream=None) -> int:
+    """Test hook: dense q.k scores [H, N, N] of one small graph through the tensor-core pipeline."""
+    N, H, d = Q.shape
+    return int(lib().kmip_debug_tc_scores(_ptr(Q), _ptr(K), N, H, d, _ptr(scores), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+# ------------------------------------------------------------------------------------------------
+# Buffer helpers (allocation only)
+# ------------------------------------------------------------------------------------------------
+def storage_dtype(mode: int):
+    return torch.bfloat16 if mode == KMIP_BF16_TC else torch.float32
+
+
+class ForwardBuffers:
+    """Outputs and scratch of one forward problem size, allocated once with torch."""
+
+    def __init__(self, N, G, H, d, k, mode, device="cuda"):
+        dt = storage_dtype(mode)
+        self.out = torch.empty((N, H, d), dtype=dt, device=device)
+        self.topk_idx = torch.empty((N, H, k), dtype=torch.int32, device=device)
+        self.topk_score = torch.empty((N, H, k), dtype=torch.float32, device=device)
+        nbytes = kmip_attn_workspace_bytes(N, G, H, d, k, mode, PASS_FORWARD)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+class BackwardBuffers:
+    """Gradients and scratch of one backward problem size, allocated once with torch."""
+
+    def __init__(self, N, G, H, d, k, mode, device="cuda"):
+        dt = storage_dtype(mode)
+        self.dQ = torch.empty((N, H, d), dtype=dt, device=device)
+        self.dK = torch.empty((N, H, d), dtype=dt, device=device)
+        self.dV = torch.empty((N, H, d), dtype=dt, device=device)
+        nbytes = kmip_attn_workspace_bytes(N, G, H, d, k, mode, PASS_BACKWARD)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def forward(Q, K, V, graph_offsets, k, mode, buffers: ForwardBuffers | None = None, stream=None, check=True):
+    """Allocate (unless given) and run the forward pass; returns the buffers."""
+    N, H, d = Q.shape
+    G = 1 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    b = buffers or ForwardBuffers(N, G, H, d, k, mode, Q.device)
+    rc = kmip_attn_forward(Q, K, V, graph_offsets, k, mode, b.out, b.topk_idx, b.topk_score, b.workspace, stream)
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_attn_forward")
+    if check:
+        st = kmip_last_status(b.workspace, stream)
+        if st != KMIP_OK:
+            raise KmipError(st, "kmip_attn_forward (device)")
+    return b
+
+
+def backward(Q, K, V, graph_offsets, k, mode, fwd: ForwardBuffers, d_out,
+             buffers: BackwardBuffers | None = None, stream=None, check=True):
+    """Allocate (unless given) and run the backward pass; returns the buffers."""
+    N, H, d = Q.shape
+    G = 1 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    b = buffers or BackwardBuffers(N, G, H, d, k, mode, Q.device)
+    rc = kmip_attn_backward(Q, K, V, graph_offsets, k, mode, fwd.out, d_out, fwd.topk_idx, fwd.topk_score,
+                            b.dQ, b.dK, b.dV, b.workspace, stream)
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_attn_backward")
+    if check:
+        st = kmip_last_status(b.workspace, stream)
+        if st != KMIP_OK:
+            raise KmipError(st, "kmip_attn_backward (device)")
+    return b

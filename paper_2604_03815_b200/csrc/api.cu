@@ -1,0 +1,125 @@
+// C ABI of the k-MIP attention library: argument validation and kernel sequencing.
+// Nothing here allocates device memory or synchronises the stream (kmip_last_status excepted).
+#include "common.cuh"
+
+using namespace kmip;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int64_t N, int32_t H, int32_t d, int32_t k, int mode) {
+    if (N < 0 || N >= (int64_t)1 << 31 || H < 1 || k < 1 || d < 1) return KMIP_ERR_INVALID_ARG;
+    if (mode != KMIP_BF16_TC && mode != KMIP_FP32_EXACT) return KMIP_ERR_UNSUPPORTED;
+    if (d != 16 && d != 32 && d != 64 && d != 128) return KMIP_ERR_UNSUPPORTED;
+    if (k > 128) return KMIP_ERR_UNSUPPORTED;
+    if ((__int128)N * H * k >= (__int128)1 << 31) return KMIP_ERR_INVALID_ARG;
+    if ((__int128)N * H * d >= (__int128)1 << 40) return KMIP_ERR_INVALID_ARG;
+    return KMIP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int kmip_version(void) { return 100; }
+
+const char* kmip_status_string(int status) {
+    switch (status) {
+        case KMIP_OK: return "ok";
+        case KMIP_ERR_INVALID_ARG: return "invalid argument";
+        case KMIP_ERR_UNSUPPORTED: return "unsupported head width, k or mode";
+        case KMIP_ERR_WORKSPACE: return "workspace too small";
+        case KMIP_ERR_CUDA: return "CUDA runtime or launch failure";
+        case KMIP_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case KMIP_ERR_BAD_OFFSETS: return "graph_offsets is not a valid CSR offset array";
+        default: return "unknown status";
+    }
+}
+
+int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k, int mode, int pass,
+                              size_t* bytes) {
+    if (!bytes || G < 0) return KMIP_ERR_INVALID_ARG;
+    const int rc = check_shape(N, H, d, k, mode);
+    if (rc != KMIP_OK) return rc;
+    if (pass == KMIP_PASS_FORWARD) *bytes = plan_fwd_workspace(N, G).total;
+    else if (pass == KMIP_PASS_BACKWARD) *bytes = plan_bwd_workspace(N, H, k).total;
+    else return KMIP_ERR_INVALID_ARG;
+    return KMIP_OK;
+}
+
+int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
+                      int64_t N, int32_t H, int32_t d, int32_t k, int mode, void* out, int32_t* topk_idx,
+                      float* topk_score, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_shape(N, H, d, k, mode);
+    if (rc != KMIP_OK) return rc;
+    if (N == 0) return KMIP_OK;
+    if (graph_offsets != nullptr && G < 1) return KMIP_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !out || !topk_idx || !topk_score || !workspace) return KMIP_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || !aligned16(topk_idx) ||
+        !aligned16(topk_score) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
+        return KMIP_ERR_INVALID_ARG;
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1);
+    if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
+
+    FwdArgs a{Q, K, V, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, out, topk_idx, topk_score,
+              static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    const bool tc = mode == KMIP_BF16_TC && score_select_tc_supported(d, k);
+    if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 256) != cudaSuccess) return KMIP_ERR_CUDA;
+    const cudaError_t e1 = tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a);
+    if (e1 != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
+    return KMIP_OK;
+}
+
+int kmip_attn_backward(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
+                       int64_t N, int32_t H, int32_t d, int32_t k, int mode, const void* out, const void* d_out,
+                       const int32_t* topk_idx, const float* topk_score, void* dQ, void* dK, void* dV,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    (void)graph_offsets; (void)G; (void)out;
+    const int rc = check_shape(N, H, d, k, mode);
+    if (rc != KMIP_OK) return rc;
+    if (N == 0) return KMIP_OK;
+    if (!Q || !K || !V || !d_out || !topk_idx || !topk_score || !dQ || !dK || !dV || !workspace)
+        return KMIP_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(d_out) || !aligned16(topk_idx) ||
+        !aligned16(topk_score) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(workspace))
+        return KMIP_ERR_INVALID_ARG;
+    const BwdWorkspace w = plan_bwd_workspace(N, H, k);
+    if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
+    BwdArgs a{Q, K, V, d_out, N, H, d, k, mode, topk_idx, topk_score, dQ, dK, dV,
+              static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_backward(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    return KMIP_OK;
+}
+
+int kmip_last_status(const void* workspace, void* stream, int* device_status) {
+    if (!workspace || !device_status) return KMIP_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;
+    int st = 0;
+    if (cudaMemcpy(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return KMIP_ERR_CUDA;
+    *device_status = st;
+    return KMIP_OK;
+}
+
+// ---- test hook (not part of kmip.h): dense scores of the tensor-core pipeline -----------------
+// Writes S[h][i][j] = q_i^h . k_j^h (fp32, [H, N, N]) for ONE graph of N <= 8192 nodes through the
+// same TMA / tcgen05 path as the forward pass, so tests can check the contraction element-wise.
+int kmip_debug_tc_scores(const void* Q, const void* K, int64_t N, int32_t H, int32_t d, float* scores,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_shape(N, H, d, 1, KMIP_BF16_TC);
+    if (rc != KMIP_OK) return rc;
+    if (!Q || !K || !scores || !workspace || N < 1 || N > 8192) return KMIP_ERR_INVALID_ARG;
+    const FwdWorkspace w = plan_fwd_workspace(N, 1);
+    if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
+    FwdArgs a{Q, K, nullptr, nullptr, 1, N, H, d, 1, KMIP_BF16_TC, nullptr, nullptr, nullptr,
+              static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_plan(a, w, score_select_tc_rows_per_item(d, 1)) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_score_dump_tc(a, w, scores) != cudaSuccess) return KMIP_ERR_CUDA;
+    return KMIP_OK;
+}
+
+}  // extern "C"

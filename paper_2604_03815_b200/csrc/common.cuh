@@ -1,0 +1,173 @@
+// Shared declarations of the k-MIP attention kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kmip.h"
+
+namespace kmip {
+
+// ---------------------------------------------------------------------------------------------
+// Workspace layout.  The first 256 bytes are the status block; everything else is carved by the
+// host-side planners below with 256-byte alignment.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStatusBytes = 256;
+constexpr size_t kAlign = 256;
+
+struct StatusBlock {
+    int status;      // kmip_status_t recorded by the device (first error wins)
+    int detail;      // where it happened (kernel-specific code)
+    int n_items;     // forward: number of work items the plan kernel produced
+    int n_long;      // backward: number of long key segments
+    int reserved[60];
+};
+static_assert(sizeof(StatusBlock) == kStatusBytes, "status block size");
+
+// One unit of work of the tensor-core score kernel: up to 256 consecutive query rows of one
+// graph and that graph's key range (Eq. 1 restricted to the graph by the CSR offsets).
+struct WorkItem {
+    int row0;    // first query row
+    int nrows;   // 1..256
+    int key_lo;  // graph's first row
+    int key_hi;  // one past the graph's last row
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+struct FwdWorkspace {
+    size_t items_off;  // WorkItem[max_items]
+    size_t total;
+    int max_items;
+};
+
+inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G) {
+    FwdWorkspace w;
+    w.max_items = (int)(N / 128 + (G > 0 ? G : 1) + 1);
+    w.items_off = kStatusBytes;
+    w.total = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
+    return w;
+}
+
+struct BwdWorkspace {
+    size_t p_off;         // float [N*H*k]   softmax weights
+    size_t ds_off;        // float [N*H*k]   score gradients
+    size_t seg_off;       // int   [N*H+1]   start of each (key, head) hit list
+    size_t cursor_off;    // int   [N*H]     hit counts, then fill cursors
+    size_t pairs_off;     // int   [N*H*k]   hit lists: flat pair ids (i*H+h)*k+t
+    size_t blocksum_off;  // int   [scan blocks]
+    size_t long_off;      // int   [N*H]     ids of long segments
+    size_t total;
+    int scan_blocks;
+};
+
+constexpr int kScanItemsPerBlock = 4096;
+
+inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
+    BwdWorkspace w;
+    const size_t rows = (size_t)N * H, pairs = rows * (size_t)k;
+    w.scan_blocks = (int)((rows + 1 + kScanItemsPerBlock - 1) / kScanItemsPerBlock);
+    size_t o = kStatusBytes;
+    w.p_off = o;        o = align_up(o + 4 * pairs);
+    w.ds_off = o;       o = align_up(o + 4 * pairs);
+    w.seg_off = o;      o = align_up(o + 4 * (rows + 1));
+    w.cursor_off = o;   o = align_up(o + 4 * (rows + 1));
+    w.pairs_off = o;    o = align_up(o + 4 * pairs);
+    w.blocksum_off = o; o = align_up(o + 4 * (size_t)(w.scan_blocks + 1));
+    w.long_off = o;     o = align_up(o + 4 * rows);
+    w.total = o;
+    return w;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ inline void record_status(StatusBlock* sb, int status, int detail) {
+    if (atomicCAS(&sb->status, 0, status) == 0) sb->detail = detail;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kVec = 4;  // elements per 16-byte vector
+    __device__ static inline float load(const float* p) { return __ldg(p); }
+    __device__ static inline void store(float* p, float v) { *p = v; }
+    __device__ static inline void load_vec(const float* p, float (&v)[4]) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    __device__ static inline void store_vec(float* p, const float (&v)[4]) {
+        *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+    __device__ static inline float load(const __nv_bfloat16* p) {
+        return __uint_as_float(((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    }
+    __device__ static inline void store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+    __device__ static inline void load_vec(const __nv_bfloat16* p, float (&v)[8]) {
+        const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    __device__ static inline void store_vec(__nv_bfloat16* p, const float (&v)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&b);
+        }
+        *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Kernel launchers (defined in the .cu files; all asynchronous on `stream`)
+// ---------------------------------------------------------------------------------------------
+struct FwdArgs {
+    const void *Q, *K, *V;
+    const int32_t* graph_offsets;  // may be null
+    int32_t G;
+    int64_t N;
+    int32_t H, d, k;
+    int mode;
+    void* out;
+    int32_t* topk_idx;
+    float* topk_score;
+    unsigned char* ws;
+    cudaStream_t stream;
+};
+
+struct BwdArgs {
+    const void *Q, *K, *V, *d_out;
+    int64_t N;
+    int32_t H, d, k;
+    int mode;
+    const int32_t* topk_idx;
+    const float* topk_score;
+    void *dQ, *dK, *dV;
+    unsigned char* ws;
+    cudaStream_t stream;
+};
+
+// plan.cu: validates the offsets and writes the work items of the tensor-core kernel
+cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_item);
+// score_select_exact.cu: CUDA-core scores + running top-k, any supported (d, k), fp32 or bf16 storage
+cudaError_t launch_score_select_exact(const FwdArgs& a);
+// score_select_tc.cu: tcgen05 scores + running top-k (bf16 storage); returns cudaErrorNotSupported
+// when (d, k) is outside what the tensor-core kernel covers
+bool score_select_tc_supported(int32_t d, int32_t k);
+int score_select_tc_rows_per_item(int32_t d, int32_t k);
+cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w);
+cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump);
+// epilogue.cu: softmax over the k kept scores fused with the gather-V weighted sum
+cudaError_t launch_softmax_gather(const FwdArgs& a);
+// backward.cu
+cudaError_t launch_backward(const BwdArgs& a, const BwdWorkspace& w);
+
+}  // namespace kmip

@@ -1,0 +1,91 @@
+// Plan kernel: CSR graph offsets -> work items of the tensor-core score kernel.
+// The paper leaves open how the graphs of a batch are kept apart; here a query only ever sees
+// the key range of its own graph, so each item carries that range.  Runs on the device so the
+// host never reads graph_offsets.
+#include "common.cuh"
+
+namespace kmip {
+
+namespace {
+
+constexpr int kPlanThreads = 1024;
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(const int32_t* __restrict__ offs, int G, int N, int rows_per_item, int max_items,
+            WorkItem* __restrict__ items, StatusBlock* __restrict__ sb) {
+    __shared__ int s_warp[32];
+    __shared__ int s_carry;
+    __shared__ int s_bad;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid == 0) { s_carry = 0; s_bad = 0; }
+    __syncthreads();
+
+    if (offs != nullptr) {
+        int bad = 0;
+        if (tid == 0 && (__ldg(offs) != 0 || __ldg(offs + G) != N)) bad = 1;
+        for (int g = tid; g < G; g += kPlanThreads)
+            if (__ldg(offs + g) > __ldg(offs + g + 1) || __ldg(offs + g) < 0) bad = 1;
+        if (bad) s_bad = 1;
+        __syncthreads();
+        if (s_bad) {
+            if (tid == 0) { record_status(sb, KMIP_ERR_BAD_OFFSETS, 1); sb->n_items = 0; }
+            return;
+        }
+    }
+
+    const int n_graphs = offs ? G : 1;
+    for (int g0 = 0; g0 < n_graphs; g0 += kPlanThreads) {
+        const int g = g0 + tid;
+        int lo = 0, hi = 0;
+        if (g < n_graphs) {
+            lo = offs ? __ldg(offs + g) : 0;
+            hi = offs ? __ldg(offs + g + 1) : N;
+        }
+        const int tiles = (hi - lo + rows_per_item - 1) / rows_per_item;
+        // block-wide exclusive scan of `tiles`
+        int incl = tiles;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_warp[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            int w = s_warp[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, w, o);
+                if (lane >= o) w += t;
+            }
+            s_warp[lane] = w;  // inclusive over warps
+        }
+        __syncthreads();
+        const int base = s_carry + (wid ? s_warp[wid - 1] : 0) + incl - tiles;
+        for (int t = 0; t < tiles; ++t) {
+            if (base + t < max_items) {
+                WorkItem it;
+                it.row0 = lo + t * rows_per_item;
+                it.nrows = min(rows_per_item, hi - it.row0);
+                it.key_lo = lo;
+                it.key_hi = hi;
+                items[base + t] = it;
+            }
+        }
+        __syncthreads();
+        if (tid == 0) s_carry += s_warp[31];
+        __syncthreads();
+    }
+    if (tid == 0) sb->n_items = min(s_carry, max_items);
+}
+
+}  // namespace
+
+cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_item) {
+    plan_kernel<<<1, kPlanThreads, 0, a.stream>>>(
+        a.graph_offsets, a.G, (int)a.N, rows_per_item, w.max_items,
+        reinterpret_cast<WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws));
+    return cudaGetLastError();
+}
+
+}  // namespace kmip

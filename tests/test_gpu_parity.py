@@ -1,0 +1,156 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_03815_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2604_03815_b200 import binding as kb
+    from tests import parity_util as pu
+
+
+def _fwd_bwd(w, rows=None, backward=True):
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    st = pu.check_forward(w, fb, rows)
+    if backward:
+        bb = pu.run_backward(w, fb, dev)
+        st.update(pu.check_backward(w, fb, bb))
+    return st
+
+
+# ------------------------------------------------------------------ tensor-core contraction alone
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
+def test_tc_dense_scores_match_fp64(d):
+    N, H = 300, 2                      # three key tiles with a ragged tail, two 128-row query tiles + tail
+    w = wl.iid_workload("s", 40 + d, [N], H, d, 4, wl.MODE_BF16_TC)
+    Q, K, V, dO, offs = pu.to_device(w)
+    S = torch.full((H, N, N), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(kb.kmip_attn_workspace_bytes(N, 1, H, d, 1, kb.KMIP_BF16_TC, kb.PASS_FORWARD),
+                     dtype=torch.uint8, device="cuda")
+    assert kb.kmip_debug_tc_scores(Q, K, S, ws) == kb.KMIP_OK
+    assert kb.kmip_last_status(ws) == kb.KMIP_OK
+    ref = np.einsum("ihc,jhc->hij", w.Q.astype(np.float64), w.K.astype(np.float64))
+    got = S.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    np.testing.assert_allclose(got, ref, rtol=2e-5, atol=1e-5 * np.sqrt(d))
+
+
+# ------------------------------------------------------------------ small cases, every element
+def test_config1_fp32_exact():
+    w = wl.make_config(1)
+    st = _fwd_bwd(w, backward=False)
+    assert st["identical_rows"] == 1.0 and st["min_gap"] > pu.FP32_SCORE_ERR
+
+
+def test_config1_fp32_backward_too():
+    w = wl.make_config(1)
+    _fwd_bwd(w, backward=True)
+
+
+def test_config2_batched_small_graphs():
+    w = wl.make_config(2)
+    st = _fwd_bwd(w)
+    assert st["identical_rows"] > 0.99
+
+
+@pytest.mark.parametrize("d,k,H,N", [(32, 16, 4, 3000), (16, 8, 3, 2500), (64, 32, 2, 1500), (128, 20, 1, 1100),
+                                     (32, 1, 2, 700), (32, 32, 1, 257), (16, 48, 2, 900), (64, 96, 1, 700),
+                                     (128, 64, 1, 600), (32, 128, 1, 600)])
+def test_small_single_graph_bf16(d, k, H, N):
+    w = wl.iid_workload("s", 1000 + d + k, [N], H, d, k, wl.MODE_BF16_TC, input_scale=1.0 / np.sqrt(d))
+    st = _fwd_bwd(w)
+    assert st["identical_rows"] > 0.98
+
+
+@pytest.mark.parametrize("d,k", [(16, 5), (32, 16), (64, 40), (128, 100)])
+def test_small_fp32_mode(d, k):
+    w = wl.iid_workload("s", 2000 + d, [500, 300], 2, d, k, wl.MODE_FP32_EXACT, input_scale=1.0 / np.sqrt(d))
+    st = _fwd_bwd(w)
+    assert st["identical_rows"] == 1.0
+
+
+def test_small_pointcloud_mixture():
+    w = wl.make_config(4, N=4000)
+    _fwd_bwd(w)
+
+
+def test_small_hub_batch():
+    w = wl.make_config(5, n_per_graph=1500)
+    _fwd_bwd(w)
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("mode", [wl.MODE_BF16_TC, wl.MODE_FP32_EXACT])
+def test_ragged_batch_with_tiny_and_empty_graphs(mode):
+    sizes = [1, 0, 3, 129, 0, 7, 256, 2, 385, 16, 31, 33]
+    w = wl.iid_workload("s", 77, sizes, 2, 32, 16, mode)
+    st = _fwd_bwd(w)
+    assert st["rows"] == sum(sizes)
+
+
+def test_single_node():
+    w = wl.iid_workload("s", 78, [1], 2, 16, 4, wl.MODE_BF16_TC)
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    assert fb.topk_idx.cpu().numpy()[0, :, 0].tolist() == [0, 0]
+    assert np.all(fb.topk_idx.cpu().numpy()[0, :, 1:] == -1)
+    np.testing.assert_allclose(fb.out.float().cpu().numpy(), w.V, rtol=1e-2)
+    pu.check_forward(w, fb)
+
+
+@pytest.mark.parametrize("mode", [wl.MODE_BF16_TC, wl.MODE_FP32_EXACT])
+def test_identical_keys_tie_break_by_index(mode):
+    w = wl.iid_workload("s", 79, [200, 90], 2, 32, 8, mode)
+    w.K[:] = w.K[5]
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    idx = fb.topk_idx.cpu().numpy()
+    assert np.all(idx[:200] == np.arange(8)) and np.all(idx[200:] == 200 + np.arange(8))
+    pu.check_forward(w, fb)
+
+
+def test_null_offsets_means_one_graph():
+    w = wl.iid_workload("s", 80, [600], 2, 32, 8, wl.MODE_BF16_TC)
+    Q, K, V, dO, offs = pu.to_device(w)
+    a = kb.forward(Q, K, V, offs, w.k, w.mode)
+    b = kb.forward(Q, K, V, None, w.k, w.mode)
+    torch.cuda.synchronize()
+    assert torch.equal(a.topk_idx, b.topk_idx) and torch.equal(a.out, b.out)
+
+
+def test_forward_is_deterministic():
+    w = wl.make_config(5, n_per_graph=1200)
+    dev = pu.to_device(w)
+    a = pu.run_forward(w, dev)
+    b = pu.run_forward(w, dev)
+    assert torch.equal(a.topk_idx, b.topk_idx) and torch.equal(a.topk_score, b.topk_score) and torch.equal(a.out, b.out)
+
+
+def test_bad_offsets_are_reported_by_the_device():
+    w = wl.iid_workload("s", 81, [300, 300], 1, 32, 8, wl.MODE_BF16_TC)
+    Q, K, V, dO, offs = pu.to_device(w)
+    bad = torch.tensor([0, 400, 300, 600], dtype=torch.int32, device="cuda")
+    b = kb.ForwardBuffers(600, 3, 1, 32, 8, w.mode)
+    assert kb.kmip_attn_forward(Q, K, V, bad, 8, w.mode, b.out, b.topk_idx, b.topk_score, b.workspace) == kb.KMIP_OK
+    assert kb.kmip_last_status(b.workspace) == kb.KMIP_ERR_BAD_OFFSETS
+    # the context is still usable afterwards
+    pu.check_forward(w, pu.run_forward(w, (Q, K, V, dO, offs)))
+
+
+def test_workspace_too_small_is_refused():
+    w = wl.iid_workload("s", 82, [300], 1, 32, 8, wl.MODE_BF16_TC)
+    Q, K, V, dO, offs = pu.to_device(w)
+    b = kb.ForwardBuffers(300, 1, 1, 32, 8, w.mode)
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    assert kb.kmip_attn_forward(Q, K, V, offs, 8, w.mode, b.out, b.topk_idx, b.topk_score, small) == kb.KMIP_ERR_WORKSPACE
+
+
+def test_workspace_is_linear_in_n():
+    a = kb.kmip_attn_workspace_bytes(100_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
+    b = kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
+    assert b < 10.5 * a and b < 1_000_000 * 4 * (3 * 16 + 4) * 4 + (1 << 20)
+    assert kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_FORWARD) < (1 << 20)
