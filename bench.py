@@ -1,0 +1,312 @@
+#!/usr/bin/env python
+"""Benchmark of the k-MIP attention hot path (forward + sparse backward) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 4]
+
+One step = one forward + one backward pass over the whole synthetic workload (default: the
+500k-node point-cloud graph, H=4, d=32, k=32, bf16).  Prints ONE JSON line on rank 0.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+With N > 1 (torchrun) every rank runs an independent replica; the path has no exchange step.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2604_03815_b200 import dist as kdist  # noqa: E402
+from paper_2604_03815_b200 import workloads as wl  # noqa: E402
+
+METRIC = "k-MIP fwd+bwd query-key scores/sec at N=500k"
+UNIT = "scores/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+LAUNCHES_PER_STEP = 3 + 8   # forward: plan, score+select, softmax+gather; backward: rows, hist, 3 scan, fill, 2 segment
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def describe(w):
+    return (f"{w.name}: G={w.G} N={w.N} H={w.H} d={w.d} k={w.k} "
+            f"{'bf16 tensor-core' if w.mode == wl.MODE_BF16_TC else 'fp32 exact'} mode, seeded synthetic")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.rows.append([x.strip() for x in line.split(",")])
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()          # the exact child process started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(np.max(mx)), "power_w_median": float(np.median(pw)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and the --impl reference arm)
+# ------------------------------------------------------------------------------------------------
+def oracle_step(w, rows):
+    """One bounded oracle step: forward for the sampled query rows against all keys of their graph,
+    then the backward restricted to those rows.  Returns (seconds, scores evaluated)."""
+    from oracle import kmip_oracle as oracle
+    t0 = time.perf_counter()
+    f = oracle.forward(w.Q, w.K, w.V, w.graph_offsets, w.k, rows=rows)
+    idx = np.full((w.N, w.H, w.k), -1, dtype=np.int32)
+    idx[rows] = f["idx"]
+    oracle.backward(w.Q, w.K, w.V, w.dOut, idx)
+    dt = time.perf_counter() - t0
+    offs = w.graph_offsets.astype(np.int64)
+    g = np.searchsorted(offs, rows, side="right") - 1
+    scores = int(w.H * np.sum(offs[g + 1] - offs[g]))
+    return dt, scores
+
+
+def oracle_rows(w, per_thread):
+    from oracle import kmip_oracle as oracle
+    n = max(8, per_thread * oracle.threads())
+    return wl.sample_rows(w, n), oracle.threads()
+
+
+def run_reference(args, w):
+    rank, _, world = kdist.env_world()
+    if rank != 0:
+        return None
+    rows, cores = oracle_rows(w, 32)
+    for _ in range(args.warmup):
+        oracle_step(w, rows[: max(8, len(rows) // 8)])
+    tot_t, tot_s = 0.0, 0
+    for _ in range(args.steps):
+        dt, sc = oracle_step(w, rows)
+        tot_t += dt
+        tot_s += sc
+    value = tot_s / tot_t
+    sample = f"{len(rows)} query rows (seeded, stratified) x all keys of their graph per step, forward + backward on those rows"
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(w), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    from paper_2604_03815_b200 import binding as kb
+
+    rank, local_rank, world = kdist.init()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dt = kb.storage_dtype(w.mode)
+    host = {n: torch.from_numpy(getattr(w, n)).to(dt).pin_memory() for n in ("Q", "K", "V", "dOut")}
+    offs = torch.from_numpy(w.graph_offsets).to(dev)
+    d_in = {n: t.to(dev) for n, t in host.items()}
+    fb = kb.ForwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode, dev)
+    bb = kb.BackwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode, dev)
+    host_out = {n: torch.empty((w.N, w.H, w.d), dtype=dt).pin_memory() for n in ("out", "dQ", "dK", "dV")}
+
+    def step():
+        rc = kb.kmip_attn_forward(d_in["Q"], d_in["K"], d_in["V"], offs, w.k, w.mode, fb.out, fb.topk_idx,
+                                  fb.topk_score, fb.workspace)
+        assert rc == kb.KMIP_OK, kb.status_string(rc)
+        if w.backward:
+            rc = kb.kmip_attn_backward(d_in["Q"], d_in["K"], d_in["V"], offs, w.k, w.mode, fb.out, d_in["dOut"],
+                                       fb.topk_idx, fb.topk_score, bb.dQ, bb.dK, bb.dV, bb.workspace)
+            assert rc == kb.KMIP_OK, kb.status_string(rc)
+
+    def step_e2e():
+        for n in ("Q", "K", "V", "dOut"):
+            d_in[n].copy_(host[n], non_blocking=True)
+        step()
+        host_out["out"].copy_(fb.out, non_blocking=True)
+        if w.backward:
+            for n in ("dQ", "dK", "dV"):
+                host_out[n].copy_(getattr(bb, n), non_blocking=True)
+
+    def timed(fn, steps):
+        kdist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        kdist.barrier()
+        return e0.elapsed_time(e1) / 1e3
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
+
+    kb.kmip_profile_enable(min(args.steps, 256))
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    secs = timed(step, args.steps)
+    clocks = sampler.stop()
+    stage_ms, n_f, n_b = kb.kmip_profile_read()
+    kb.kmip_profile_enable(0)
+    assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
+
+    for _ in range(min(args.warmup, 2)):
+        step_e2e()
+    secs_e2e = timed(step_e2e, args.steps)
+
+    units = float(w.n_scores) * args.steps
+    value, t_max = kdist.aggregate_throughput(units, secs)
+    value_e2e, _ = kdist.aggregate_throughput(units, secs_e2e)
+    if rank != 0:
+        kdist.shutdown()
+        return None
+
+    peaks = load_peaks()
+    per_call = {s: (stage_ms[s] / max(1, n_f if i < 3 else n_b)) for i, s in enumerate(kb.STAGES)}
+    fwd_ms = per_call["plan"] + per_call["score_select"] + per_call["softmax_gather"]
+    bwd_ms = per_call["bwd_rows"] + per_call["bwd_inverse_index"] + per_call["bwd_segments"]
+    flops = 2.0 * w.d * w.n_scores
+    tflops = flops / (per_call["score_select"] * 1e-3) / 1e12 if per_call["score_select"] > 0 else 0.0
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "score_select_traffic.json")
+    if os.path.exists(tp):
+        with open(tp) as f:
+            tj = json.load(f)
+        if tj.get("workload") == w.name:
+            traffic = tj.get("dram_bytes_per_launch")
+    tensor_kernel = w.mode == wl.MODE_BF16_TC
+    roofline = {
+        "kernel": "score_select_tc_kernel (tcgen05 scores + running top-k)" if tensor_kernel else "score_select_exact_kernel",
+        "bound": "tensor" if tensor_kernel else "alu",
+        "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+        "frac": tflops / peaks["bf16_tflops"], "frac_of_sustained_peak": tflops / peaks["bf16_tflops_sustained"],
+        "peak_source": f"{peaks['_source']} (burst cuBLAS bf16; sustained {peaks['bf16_tflops_sustained']})",
+        "flops_per_launch": flops, "ms_per_launch": per_call["score_select"], "traffic": traffic,
+    }
+    pairs = w.N * w.H * w.k
+    esz = 2 if w.mode == wl.MODE_BF16_TC else 4
+    bwd_bytes = pairs * (4 * w.d * esz + 28) + 7 * w.N * w.H * w.d * esz
+    fwd_tail_bytes = w.N * w.H * (w.k * (8 + w.d * esz) + w.d * esz)
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.mode == wl.MODE_BF16_TC else "f32", "data": "synthetic",
+        "config": {"workload": describe(w), "passes": "forward+backward" if w.backward else "forward",
+                   "l2": "Q, K, V, dOut and the outputs (>=128 MB each) exceed the 126 MB L2; no flush between steps",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "roofline": roofline,
+        "stages_ms": {k_: round(v, 4) for k_, v in per_call.items()},
+        "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
+        "fwd_scores_per_s": w.n_scores / (fwd_ms * 1e-3) if fwd_ms > 0 else None,
+        "rows_per_s": w.N * w.H / (1e-3 * (fwd_ms + bwd_ms)) if fwd_ms + bwd_ms > 0 else None,
+        "hbm_stages": {
+            "softmax_gather_gbs": fwd_tail_bytes / (per_call["softmax_gather"] * 1e-3) / 1e9 if per_call["softmax_gather"] > 0 else None,
+            "backward_gbs": bwd_bytes / (bwd_ms * 1e-3) / 1e9 if bwd_ms > 0 else None,
+            "peak_gbs": peaks["hbm_gbs"],
+        },
+        "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": 1e3 * secs_e2e / args.steps,
+                "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host.values())),
+                "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for n, t in host_out.items()
+                                              if w.backward or n == "out"))},
+        "gpu_launches": (LAUNCHES_PER_STEP if w.backward else 3) * args.steps,
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        rows, cores = oracle_rows(w, 16)
+        dt_o, sc_o = oracle_step(w, rows)
+        result["cpu_baseline"] = {
+            "value": sc_o / dt_o, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt_o,
+            "sample": f"{len(rows)} query rows (seeded, stratified) x all keys of their graph, forward + backward on those rows",
+        }
+    kdist.shutdown()
+    return result
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", type=int, default=4, help="workload number (1-5); the headline is 4")
+    ap.add_argument("--nodes", type=int, default=0, help="override the node count of configs 3/4 (profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank, _, world = kdist.env_world()
+    if args.impl == "reference" and rank != 0:
+        return
+    kw = {"N": args.nodes} if args.nodes and args.config in (3, 4) else {}
+    w = wl.make_config(args.config, **kw)
+    res = run_reference(args, w) if args.impl == "reference" else run_ours(args, w)
+    if res is not None:
+        print(json.dumps(res), flush=True)
+
+
+if __name__ == "__main__":
+    main()

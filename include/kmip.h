@@ -116,6 +116,19 @@ int kmip_attn_backward(const void *Q, const void *K, const void *V,
  */
 int kmip_last_status(const void *workspace, void *stream, int *device_status);
 
+/*
+ * Optional per-stage timing for benchmarks; the paper has no counterpart (its Fig. 3 reports a
+ * stage breakdown measured from outside).  kmip_profile_enable(n > 0) creates CUDA events for up
+ * to n forward and n backward calls (n <= 256) and makes the two passes record them around their
+ * stages on the caller's stream; kmip_profile_enable(0) destroys them and turns recording off.
+ * kmip_profile_read waits for the recorded events, adds up the stage times in milliseconds into
+ * stage_ms[6] = {plan, score+select, softmax+gather-V, backward rows, inverse index, dK/dV
+ * segments}, stores the number of forward / backward calls recorded in calls[2] and resets the
+ * counters.  Process-wide state, not thread-safe, one device; leave it off on the hot path.
+ */
+int kmip_profile_enable(int max_calls);
+int kmip_profile_read(double *stage_ms, int *calls);
+
 /* Static, NUL-terminated description of a status code. */
 const char *kmip_status_string(int status);
 

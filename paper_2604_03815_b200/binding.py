@@ -55,6 +55,10 @@ def lib() -> ctypes.CDLL:
                                          P, P, P, P, sz, P]
         L.kmip_last_status.restype = ctypes.c_int
         L.kmip_last_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_int)]
+        L.kmip_profile_enable.restype = ctypes.c_int
+        L.kmip_profile_enable.argtypes = [ctypes.c_int]
+        L.kmip_profile_read.restype = ctypes.c_int
+        L.kmip_profile_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
         L.kmip_debug_tc_scores.restype = ctypes.c_int
         L.kmip_debug_tc_scores.argtypes = [P, P, i64, i32, i32, P, P, sz, P]
         _lib = L
@@ -115,6 +119,25 @@ def kmip_last_status(workspace, stream=None) -> int:
     if rc != KMIP_OK:
         raise KmipError(rc, "kmip_last_status")
     return int(st.value)
+
+
+STAGES = ("plan", "score_select", "softmax_gather", "bwd_rows", "bwd_inverse_index", "bwd_segments")
+
+
+def kmip_profile_enable(max_calls: int) -> None:
+    rc = lib().kmip_profile_enable(int(max_calls))
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_profile_enable")
+
+
+def kmip_profile_read():
+    """Returns ({stage: total milliseconds}, forward calls, backward calls) since the last read."""
+    ms = (ctypes.c_double * 6)()
+    calls = (ctypes.c_int * 2)()
+    rc = lib().kmip_profile_read(ms, calls)
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_profile_read")
+    return dict(zip(STAGES, list(ms))), int(calls[0]), int(calls[1])
 
 
 def kmip_debug_tc_scores(Q, K, scores, workspace, stream=None) -> int:

@@ -18,6 +18,17 @@ int check_shape(int64_t N, int32_t H, int32_t d, int32_t k, int mode) {
     return KMIP_OK;
 }
 
+// ---- optional per-stage timing (off unless kmip_profile_enable was called) ----------------------
+constexpr int kProfMaxCalls = 256;
+struct Profile {
+    bool on = false;
+    int max_calls = 0;
+    int n_fwd = 0, n_bwd = 0;
+    cudaEvent_t fwd[kProfMaxCalls][4];
+    cudaEvent_t bwd[kProfMaxCalls][4];
+};
+Profile g_prof;
+
 }  // namespace
 
 extern "C" {
@@ -65,11 +76,16 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     FwdArgs a{Q, K, V, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, out, topk_idx, topk_score,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
+    if (ev) cudaEventRecord(ev[0], a.stream);
     const bool tc = mode == KMIP_BF16_TC && score_select_tc_supported(d, k);
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 256) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[1], a.stream);
     const cudaError_t e1 = tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a);
     if (e1 != cudaSuccess) return KMIP_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[2], a.stream);
     if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[3], a.stream);
     return KMIP_OK;
 }
 
@@ -91,7 +107,9 @@ int kmip_attn_backward(const void* Q, const void* K, const void* V, const int32_
     BwdArgs a{Q, K, V, d_out, N, H, d, k, mode, topk_idx, topk_score, dQ, dK, dV,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
-    if (launch_backward(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    cudaEvent_t* ev = (g_prof.on && g_prof.n_bwd < g_prof.max_calls) ? g_prof.bwd[g_prof.n_bwd++] : nullptr;
+    if (ev) cudaEventRecord(ev[0], a.stream);
+    if (launch_backward(a, w, ev ? ev + 1 : nullptr) != cudaSuccess) return KMIP_ERR_CUDA;
     return KMIP_OK;
 }
 
@@ -101,6 +119,47 @@ int kmip_last_status(const void* workspace, void* stream, int* device_status) {
     int st = 0;
     if (cudaMemcpy(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return KMIP_ERR_CUDA;
     *device_status = st;
+    return KMIP_OK;
+}
+
+int kmip_profile_enable(int max_calls) {
+    if (g_prof.on) {
+        for (int i = 0; i < g_prof.max_calls; ++i)
+            for (int e = 0; e < 4; ++e) { cudaEventDestroy(g_prof.fwd[i][e]); cudaEventDestroy(g_prof.bwd[i][e]); }
+        g_prof.on = false;
+    }
+    g_prof.n_fwd = g_prof.n_bwd = 0;
+    g_prof.max_calls = 0;
+    if (max_calls <= 0) return KMIP_OK;
+    if (max_calls > kProfMaxCalls) max_calls = kProfMaxCalls;
+    for (int i = 0; i < max_calls; ++i)
+        for (int e = 0; e < 4; ++e)
+            if (cudaEventCreate(&g_prof.fwd[i][e]) != cudaSuccess || cudaEventCreate(&g_prof.bwd[i][e]) != cudaSuccess)
+                return KMIP_ERR_CUDA;
+    g_prof.max_calls = max_calls;
+    g_prof.on = true;
+    return KMIP_OK;
+}
+
+int kmip_profile_read(double* stage_ms, int* calls) {
+    if (!stage_ms || !calls) return KMIP_ERR_INVALID_ARG;
+    for (int s = 0; s < 6; ++s) stage_ms[s] = 0.0;
+    calls[0] = g_prof.n_fwd;
+    calls[1] = g_prof.n_bwd;
+    if (!g_prof.on) return KMIP_OK;
+    for (int pass = 0; pass < 2; ++pass) {
+        const int n = pass ? g_prof.n_bwd : g_prof.n_fwd;
+        for (int i = 0; i < n; ++i) {
+            cudaEvent_t* ev = pass ? g_prof.bwd[i] : g_prof.fwd[i];
+            if (cudaEventSynchronize(ev[3]) != cudaSuccess) return KMIP_ERR_CUDA;
+            for (int s = 0; s < 3; ++s) {
+                float ms = 0.0f;
+                if (cudaEventElapsedTime(&ms, ev[s], ev[s + 1]) != cudaSuccess) return KMIP_ERR_CUDA;
+                stage_ms[pass * 3 + s] += ms;
+            }
+        }
+    }
+    g_prof.n_fwd = g_prof.n_bwd = 0;
     return KMIP_OK;
 }
 

@@ -35,7 +35,7 @@ bwd_rows_kernel(const T* __restrict__ K, const T* __restrict__ V, const T* __res
         const int h = (int)(r % H);
         int j[kMaxEntriesPerLane];
         float p[kMaxEntriesPerLane];
-        load_row_softmax(topk_idx + (size_t)r * k, topk_score + (size_t)r * k, k, scale, lane, j, p);
+        load_row_softmax(topk_idx + (size_t)r * k, topk_score + (size_t)r * k, k, N, scale, lane, j, p);
 
         // dP_t = g_i . v_{j_t}: each lane owns its entries and walks the d columns
         float dP[kMaxEntriesPerLane];
@@ -323,7 +323,7 @@ bwd_long_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
 
 // -------------------------------------------------------------------------------------- launcher
 template <typename T, int D>
-cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w) {
+cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     const long long n_rows = (long long)a.N * a.H, n_pairs = n_rows * a.k;
     StatusBlock* sb = reinterpret_cast<StatusBlock*>(a.ws);
     float* ws_p = reinterpret_cast<float*>(a.ws + w.p_off);
@@ -343,6 +343,7 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w) {
     const int row_blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
     bwd_rows_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         K, V, dOut, a.topk_idx, a.topk_score, (int)a.N, a.H, a.k, scale, ws_p, ws_ds, static_cast<T*>(a.dQ));
+    if (ev) cudaEventRecord(ev[0], a.stream);
 
     const int pair_blocks = (int)((n_pairs + 255) / 256);
     hist_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, cursor);
@@ -350,29 +351,31 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w) {
     scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(block_sums, w.scan_blocks);
     scan_write_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums, seg_off, long_list, sb);
     fill_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, seg_off, cursor, pairs);
+    if (ev) cudaEventRecord(ev[1], a.stream);
 
     bwd_segments_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         Q, dOut, ws_p, ws_ds, seg_off, pairs, n_rows, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
     bwd_long_segments_kernel<T, D><<<148 * 4, kWarpsPerBlock * 32, 0, a.stream>>>(
         Q, dOut, ws_p, ws_ds, seg_off, pairs, long_list, sb, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
+    if (ev) cudaEventRecord(ev[2], a.stream);
     return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t launch_t(const BwdArgs& a, const BwdWorkspace& w) {
+cudaError_t launch_t(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     switch (a.d) {
-        case 16: return launch_d<T, 16>(a, w);
-        case 32: return launch_d<T, 32>(a, w);
-        case 64: return launch_d<T, 64>(a, w);
-        case 128: return launch_d<T, 128>(a, w);
+        case 16: return launch_d<T, 16>(a, w, ev);
+        case 32: return launch_d<T, 32>(a, w, ev);
+        case 64: return launch_d<T, 64>(a, w, ev);
+        case 128: return launch_d<T, 128>(a, w, ev);
         default: return cudaErrorInvalidValue;
     }
 }
 
 }  // namespace
 
-cudaError_t launch_backward(const BwdArgs& a, const BwdWorkspace& w) {
-    return a.mode == KMIP_FP32_EXACT ? launch_t<float>(a, w) : launch_t<__nv_bfloat16>(a, w);
+cudaError_t launch_backward(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
+    return a.mode == KMIP_FP32_EXACT ? launch_t<float>(a, w, ev) : launch_t<__nv_bfloat16>(a, w, ev);
 }
 
 }  // namespace kmip

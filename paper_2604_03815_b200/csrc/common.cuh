@@ -168,6 +168,7 @@ cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float*
 // epilogue.cu: softmax over the k kept scores fused with the gather-V weighted sum
 cudaError_t launch_softmax_gather(const FwdArgs& a);
 // backward.cu
-cudaError_t launch_backward(const BwdArgs& a, const BwdWorkspace& w);
+// ev (optional): three events recorded after the rows, inverse-index and segment stages
+cudaError_t launch_backward(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev);
 
 }  // namespace kmip

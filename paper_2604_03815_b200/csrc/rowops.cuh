@@ -23,8 +23,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Entry t of a row lives in lane t%32, register t/32.  Loads the row's indices and scores and
 // turns the scores into softmax weights p_t = exp((s_t - max)/sqrt(d)) / sum (Algorithm 1 line 5).
-// Empty slots (index < 0) get weight 0.
-__device__ __forceinline__ void load_row_softmax(const int32_t* idx_row, const float* score_row, int k,
+// Empty slots (index < 0) and indices outside [0, N) get weight 0.
+__device__ __forceinline__ void load_row_softmax(const int32_t* idx_row, const float* score_row, int k, int N,
                                                  float scale, int lane,
                                                  int (&j)[kMaxEntriesPerLane], float (&p)[kMaxEntriesPerLane]) {
     float m = -CUDART_INF_F;
@@ -35,6 +35,7 @@ __device__ __forceinline__ void load_row_softmax(const int32_t* idx_row, const f
         p[e] = -CUDART_INF_F;
         if (t < k) {
             j[e] = __ldg(idx_row + t);
+            if (j[e] >= N) j[e] = -1;  // never follow an index outside the batch
             const float s = __ldg(score_row + t);
             if (j[e] >= 0) p[e] = s;
         }

@@ -31,7 +31,9 @@ template <typename T, int D, int E>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 score_select_exact_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                           const int32_t* __restrict__ offs, int G, int N, int H, int k,
-                          int32_t* __restrict__ topk_idx, float* __restrict__ topk_score) {
+                          int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
+                          const StatusBlock* __restrict__ sb) {
+    if (sb->status != KMIP_OK) return;  // the plan kernel rejected the offsets
     constexpr int CAP = 32 * E;
     constexpr int VEC = Elem<T>::kVec;
     __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
@@ -96,7 +98,8 @@ cudaError_t launch_d(const FwdArgs& a) {
     // pending room CAP-k must hold one 32-key step beyond the compaction trigger
 #define KMIP_LAUNCH_EXACT(E_) \
     score_select_exact_kernel<T, D, E_><<<grid, block, 0, a.stream>>>( \
-        Q, K, a.graph_offsets, a.G, (int)a.N, a.H, a.k, a.topk_idx, a.topk_score)
+        Q, K, a.graph_offsets, a.G, (int)a.N, a.H, a.k, a.topk_idx, a.topk_score, \
+        reinterpret_cast<const StatusBlock*>(a.ws))
     if (a.k <= 16) KMIP_LAUNCH_EXACT(2);
     else if (a.k <= 96) KMIP_LAUNCH_EXACT(4);
     else KMIP_LAUNCH_EXACT(8);

@@ -2,7 +2,7 @@
 the same seeded inputs, compare.  Tolerances (stated once, used everywhere):
 
   fp32 mode   topk_idx bit-exact against the oracle on every row whose selection margin
-              (k-th kept score minus best excluded score) exceeds FP32_SCORE_ERR; rows below it
+              (k-th kept score minus best excluded score) exceeds FP32_SCORE_ERR*max(1,|k-th|); rows below it
               are ties at fp32 resolution and are only required to satisfy the bf16-mode rule.
   bf16 mode   every selected key's exact (oracle, fp64) score >= oracle k-th score - 1e-2*|k-th|;
               indices distinct and inside the query's own graph; padding exactly where n_g < k.
@@ -19,7 +19,7 @@ from paper_2604_03815_b200 import binding as kb
 
 OUT_ATOL, OUT_RTOL = 2e-3, 1e-2
 SCORE_ATOL, SCORE_RTOL = 1e-5, 2e-5
-FP32_SCORE_ERR = 1e-5
+FP32_SCORE_ERR = 2e-6   # relative to max(1, |k-th score|): a few fp32 ulps of a d-term sum
 SEL_RTOL = 1e-2
 
 
@@ -53,14 +53,14 @@ def check_forward(w, fb, rows=None):
     lo, hi = offs[g], offs[g + 1]
     keff = np.minimum(w.k, hi - lo)
     slot = np.arange(w.k)[None, None, :]
-    valid = slot < keff[:, None, None]
+    valid = np.broadcast_to(slot < keff[:, None, None], idx.shape)
     assert np.all(idx[~valid] == -1), "padded slots must hold -1"
     assert np.all(np.isneginf(score[~valid])), "padded slots must hold -inf"
     assert np.all((idx >= lo[:, None, None]) & (idx < hi[:, None, None]) | ~valid), "index outside the query's graph"
     srt = np.sort(np.where(valid, idx, -1 - slot), axis=-1)
     assert np.all(np.diff(srt, axis=-1) != 0), "duplicate key in a row"
     sc = np.where(valid, score, 0.0)
-    assert np.all(np.diff(np.where(valid, score, -np.inf), axis=-1) <= 0), "scores must be listed in descending order"
+    assert np.all(np.diff(np.where(valid, score, -1e300), axis=-1) <= 0), "scores must be listed in descending order"
 
     # exact scores of the keys the GPU selected, and the output the oracle derives from that set
     ref_out, exact = oracle.forward_given_idx(w.Q, w.K, w.V, idx, rows=rows)
@@ -74,7 +74,7 @@ def check_forward(w, fb, rows=None):
 
     same = np.all(idx == ref["idx"], axis=-1)
     if w.mode == kb.KMIP_FP32_EXACT:
-        decided = ref["gap"] > FP32_SCORE_ERR
+        decided = ref["gap"] > FP32_SCORE_ERR * np.maximum(1.0, np.abs(kth))
         assert np.all(same | ~decided), f"fp32 mode: topk_idx differs on {int((~same & decided).sum())} decided rows"
     d = np.abs(out - ref_out)
     assert np.all(d <= OUT_ATOL + OUT_RTOL * np.abs(ref_out)), f"out off by {d.max():.3e}"
