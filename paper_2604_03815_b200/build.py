@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libkmip.so")
-SOURCES = ["api.cu", "plan.cu", "score_select_exact.cu", "score_select_tc.cu", "epilogue.cu", "backward.cu"]
+SOURCES = ["api.cu", "plan.cu", "score_select_exact.cu", "score_select_tc.cu", "refine.cu", "epilogue.cu", "backward.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
@@ -28,6 +28,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     os.makedirs(OBJ, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
+    if os.environ.get("KMIP_SWEEP_DEBUG") == "1":   # timing experiments of the sweep kernel (developer builds)
+        extra.append("-DKMIP_SWEEP_DEBUG=1")
 
     def compile_one(src):
         obj = os.path.join(OBJ, src.replace(".cu", ".o"))

@@ -53,7 +53,8 @@ int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_
     if (!bytes || G < 0) return KMIP_ERR_INVALID_ARG;
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
-    if (pass == KMIP_PASS_FORWARD) *bytes = plan_fwd_workspace(N, G).total;
+    if (pass == KMIP_PASS_FORWARD)
+        *bytes = plan_fwd_workspace(N, G, H, d, mode == KMIP_BF16_TC && score_select_tc_supported(d, k)).total;
     else if (pass == KMIP_PASS_BACKWARD) *bytes = plan_bwd_workspace(N, H, k).total;
     else return KMIP_ERR_INVALID_ARG;
     return KMIP_OK;
@@ -70,7 +71,8 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || !aligned16(topk_idx) ||
         !aligned16(topk_score) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
         return KMIP_ERR_INVALID_ARG;
-    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1);
+    const bool tc = mode == KMIP_BF16_TC && score_select_tc_supported(d, k);
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, tc);
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
 
     FwdArgs a{Q, K, V, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, out, topk_idx, topk_score,
@@ -78,10 +80,11 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
-    const bool tc = mode == KMIP_BF16_TC && score_select_tc_supported(d, k);
+    if (tc && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 256) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
-    const cudaError_t e1 = tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a);
+    cudaError_t e1 = tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a);
+    if (e1 == cudaSuccess && tc) e1 = launch_refine_topk(a);
     if (e1 != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], a.stream);
     if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
@@ -163,6 +166,10 @@ int kmip_profile_read(double* stage_ms, int* calls) {
     return KMIP_OK;
 }
 
+// ---- timing experiments (not part of kmip.h): see set_score_select_debug_flags
+void kmip_debug_set_flags(int flags) { set_score_select_debug_flags(flags); }
+void kmip_debug_set_timing(void* buf) { set_score_select_debug_timing(static_cast<long long*>(buf)); }
+
 // ---- test hook (not part of kmip.h): dense scores of the tensor-core pipeline -----------------
 // Writes S[h][i][j] = q_i^h . k_j^h (fp32, [H, N, N]) for ONE graph of N <= 8192 nodes through the
 // same TMA / tcgen05 path as the forward pass, so tests can check the contraction element-wise.
@@ -171,11 +178,12 @@ int kmip_debug_tc_scores(const void* Q, const void* K, int64_t N, int32_t H, int
     const int rc = check_shape(N, H, d, 1, KMIP_BF16_TC);
     if (rc != KMIP_OK) return rc;
     if (!Q || !K || !scores || !workspace || N < 1 || N > 8192) return KMIP_ERR_INVALID_ARG;
-    const FwdWorkspace w = plan_fwd_workspace(N, 1);
+    const FwdWorkspace w = plan_fwd_workspace(N, 1, H, d, true);
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
     FwdArgs a{Q, K, nullptr, nullptr, 1, N, H, d, 1, KMIP_BF16_TC, nullptr, nullptr, nullptr,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_plan(a, w, score_select_tc_rows_per_item(d, 1)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_score_dump_tc(a, w, scores) != cudaSuccess) return KMIP_ERR_CUDA;
     return KMIP_OK;

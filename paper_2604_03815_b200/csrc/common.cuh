@@ -38,15 +38,18 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a = kAlign) { return
 
 struct FwdWorkspace {
     size_t items_off;  // WorkItem[max_items]
+    size_t kpack_off;  // bf16 [H, N, d]: K regrouped by head for the tensor-core sweep (0 bytes otherwise)
     size_t total;
     int max_items;
 };
 
-inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G) {
+// `tc`: the tensor-core sweep will run (bf16 mode and a supported (d, k))
+inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, bool tc) {
     FwdWorkspace w;
     w.max_items = (int)(N / 128 + (G > 0 ? G : 1) + 1);
     w.items_off = kStatusBytes;
-    w.total = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
+    w.kpack_off = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
+    w.total = align_up(w.kpack_off + (tc ? (size_t)N * H * d * 2 : 0));
     return w;
 }
 
@@ -157,14 +160,20 @@ struct BwdArgs {
 
 // plan.cu: validates the offsets and writes the work items of the tensor-core kernel
 cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_item);
+// plan.cu: K [N, H, d] -> [H, N, d] so that a head's key tile is one contiguous block for TMA
+cudaError_t launch_pack_keys(const FwdArgs& a, const FwdWorkspace& w);
 // score_select_exact.cu: CUDA-core scores + running top-k, any supported (d, k), fp32 or bf16 storage
 cudaError_t launch_score_select_exact(const FwdArgs& a);
 // score_select_tc.cu: tcgen05 scores + running top-k (bf16 storage); returns cudaErrorNotSupported
 // when (d, k) is outside what the tensor-core kernel covers
 bool score_select_tc_supported(int32_t d, int32_t k);
 int score_select_tc_rows_per_item(int32_t d, int32_t k);
+void set_score_select_debug_flags(int flags);
+void set_score_select_debug_timing(long long* buf);
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump);
+// refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k
+cudaError_t launch_refine_topk(const FwdArgs& a);
 // epilogue.cu: softmax over the k kept scores fused with the gather-V weighted sum
 cudaError_t launch_softmax_gather(const FwdArgs& a);
 // backward.cu

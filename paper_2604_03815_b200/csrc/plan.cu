@@ -79,7 +79,27 @@ plan_kernel(const int32_t* __restrict__ offs, int G, int N, int rows_per_item, i
     if (tid == 0) sb->n_items = min(s_carry, max_items);
 }
 
+// K [N, H, d] -> [H, N, d], 16 bytes per thread.
+__global__ void pack_keys_kernel(const uint4* __restrict__ K, uint4* __restrict__ Kp, long long n_vec, int N, int H,
+                                 int vec_per_row) {
+    const long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= n_vec) return;
+    const long long rowh = v / vec_per_row;  // j * H + h
+    const int c = (int)(v % vec_per_row);
+    const long long j = rowh / H;
+    const int h = (int)(rowh % H);
+    Kp[((long long)h * N + j) * vec_per_row + c] = __ldg(K + v);
+}
+
 }  // namespace
+
+cudaError_t launch_pack_keys(const FwdArgs& a, const FwdWorkspace& w) {
+    const int vec_per_row = a.d * 2 / 16;
+    const long long n_vec = (long long)a.N * a.H * vec_per_row;
+    pack_keys_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, a.stream>>>(
+        static_cast<const uint4*>(a.K), reinterpret_cast<uint4*>(a.ws + w.kpack_off), n_vec, (int)a.N, a.H, vec_per_row);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_item) {
     plan_kernel<<<1, kPlanThreads, 0, a.stream>>>(

@@ -1,0 +1,141 @@
+// Rescoring kernel of the tensor-core path (second half of Algorithm 1 line 3).
+//
+// The sweep kernel leaves, for every (query, head), the k best 8-key groups: topk_idx holds each
+// group's first key, topk_score its maximum (tensor-core score).  Those groups contain the k best
+// keys, so this kernel scores the 8k keys of a row again - fp32 fused multiply-adds over the
+// bf16 values, in index order - keeps the k best under (score desc, key asc) with the same
+// running top-k buffer as the CUDA-core kernel, and overwrites topk_idx / topk_score with them.
+// One warp per (query, head); one candidate key per lane and step.
+#include <algorithm>
+
+#include "common.cuh"
+#include "topk_buffer.cuh"
+
+namespace kmip {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kGroup = 8;  // keys per group, fixed by the sweep kernel
+
+__device__ inline int graph_end(const int32_t* offs, int G, int N, int i) {
+    if (offs == nullptr) return N;
+    int a = 0, b = G;
+    while (b - a > 1) {
+        const int m = (a + b) >> 1;
+        if (__ldg(offs + m) <= i) a = m; else b = m;
+    }
+    return max(0, min(N, __ldg(offs + a + 1)));
+}
+
+template <typename T, int D, int E>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ K, const int32_t* __restrict__ offs, int G,
+                   int N, int H, int k, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
+                   const StatusBlock* __restrict__ sb) {
+    if (sb->status != KMIP_OK) return;
+    constexpr int CAP = 32 * E;
+    constexpr int VEC = Elem<T>::kVec;
+    __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
+    __shared__ float s_q[kWarpsPerBlock][D];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    cand_t* row = s_rows[wib];
+    float* q = s_q[wib];
+    const long long n_rows = (long long)N * H;
+    const int room = CAP - k;
+
+    for (long long r = (long long)blockIdx.x * kWarpsPerBlock + wib; r < n_rows;
+         r += (long long)gridDim.x * kWarpsPerBlock) {
+        const int i = (int)(r / H), h = (int)(r % H);
+        const int hi = graph_end(offs, G, N, i);
+
+        // the row's groups: entry t in lane t%32, register t/32
+        int gid[4];
+        float theta = CUDART_INF_F;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int t = e * 32 + lane;
+            gid[e] = -1;
+            if (t < k) {
+                gid[e] = topk_idx[(size_t)r * k + t];
+                const float gmax = topk_score[(size_t)r * k + t];
+                theta = fminf(theta, gid[e] >= 0 ? gmax : -CUDART_INF_F);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) theta = fminf(theta, __shfl_xor_sync(0xFFFFFFFFu, theta, o));
+        // every key of the answer scores at least theta (the k-th best group maximum) up to the
+        // difference between tensor-core and fp32 accumulation; keep a margin for that
+        const float floor_tau = theta - 1e-4f * fabsf(theta) - 1e-30f;
+
+        __syncwarp();
+        for (int c = lane; c < D; c += 32) q[c] = Elem<T>::load(Q + ((size_t)i * H + h) * D + c);
+        for (int t = lane; t < k; t += 32) row[t] = 0ull;
+        __syncwarp();
+
+        float tau = floor_tau;
+        int cnt = 0;
+        for (int t0 = 0; t0 < k; t0 += 32 / kGroup) {
+            const int t = t0 + lane / kGroup;
+            int g = -1;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (e == (t0 >> 5)) g = __shfl_sync(0xFFFFFFFFu, gid[e], t & 31);
+            const int j = g + (lane % kGroup);
+            const bool valid = t < k && g >= 0 && j < hi;
+            float s = 0.0f;
+            if (valid) {
+                const T* kr = K + ((size_t)j * H + h) * D;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += VEC) {
+                    float kv[VEC];
+                    Elem<T>::load_vec(kr + c0, kv);
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) s = fmaf(q[c0 + c], kv[c], s);
+                }
+            }
+            const bool pass = valid && (s > tau);
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, pass);
+            if (m) {
+                if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, j);
+                cnt += __popc(m);
+                if (cnt > room - 32) {
+                    tau = fmaxf(floor_tau, warp_compact_row<E>(row, k, cnt, lane));
+                    cnt = 0;
+                }
+            }
+        }
+        warp_compact_row<E>(row, k, cnt, lane);
+        warp_store_row(row, k, lane, topk_idx + (size_t)r * k, topk_score + (size_t)r * k);
+    }
+}
+
+template <int D>
+cudaError_t launch_d(const FwdArgs& a) {
+    using T = __nv_bfloat16;
+    const long long n_rows = (long long)a.N * a.H;
+    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
+#define KMIP_LAUNCH_REFINE(E_) \
+    refine_topk_kernel<T, D, E_><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
+        static_cast<const T*>(a.Q), static_cast<const T*>(a.K), a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
+        a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws))
+    if (a.k <= 32) KMIP_LAUNCH_REFINE(2);
+    else if (a.k <= 96) KMIP_LAUNCH_REFINE(4);
+    else KMIP_LAUNCH_REFINE(8);
+#undef KMIP_LAUNCH_REFINE
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_refine_topk(const FwdArgs& a) {
+    switch (a.d) {
+        case 16: return launch_d<16>(a);
+        case 32: return launch_d<32>(a);
+        case 64: return launch_d<64>(a);
+        case 128: return launch_d<128>(a);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace kmip

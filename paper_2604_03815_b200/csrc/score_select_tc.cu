@@ -6,15 +6,27 @@
 // graph and one head, streams that graph's keys in 128-key tiles through a TMA -> shared memory
 // ring, multiplies each tile against both query tiles with tcgen05.mma (bf16 in, fp32
 // accumulators in tensor memory, double buffered), and eight selection warps read the
-// accumulators straight out of tensor memory.  One thread owns one query row: it reduces 32
-// scores to their maximum with three-input max instructions, compares once against the row's
-// threshold, and only on a hit rescans and appends candidates to the row's buffer in shared
-// memory (topk_buffer.cuh).  The N x N scores never leave the SM.
+// accumulators straight out of tensor memory.  One thread owns one query row.
+//   fast pass   the thread pulls its 128 scores of the tile into registers (the accumulator
+//               buffer goes straight back to the MMA issuer), reduces every 8 consecutive
+//               columns to their maximum with three-input max instructions and compares the
+//               tile maximum once against the row's threshold tau;
+//   candidates  a candidate is an 8-key GROUP, ranked by its maximum.  The k best groups under
+//               (maximum desc, first key asc) always contain the k best keys under (score desc,
+//               key asc): if a key of the top k sat in a group outside the best k groups, each
+//               of those k groups would hold a key that beats it.  So the sweep only tracks
+//               groups: a lane whose tile maximum beats tau appends (group maximum, first key)
+//               for the groups above tau to its pending slots - no index search, no votes;
+//   flush       when a pending area is half full all 32 lanes insert their pending groups into
+//               their own unsorted k-entry lists in lock step (replace the list minimum, 8-slot
+//               blocks with cached minima) and refresh tau = k-th best group maximum so far.
+// When an item ends each row's k groups go to global memory; refine.cu rescores their 8k keys
+// exactly and keeps the best k.  The N x N scores never leave the SM.
 //
 // Warp roles (NQT = query tiles per CTA, 1 or 2):
 //   warps 0 .. 4*NQT-1   selection; warp w reads TMEM lanes 32*(w%4).. of query tile w/4
 //   warp 4*NQT           TMA producer (one lane)
-//   warp 4*NQT+1         TMEM allocation + tcgen05.mma issue (one lane)
+//   warps 4*NQT+1, +2    tcgen05.mma issue (one lane each, alternating key tiles); +1 owns TMEM
 // Every wait is bounded; on expiry the CTA records KMIP_ERR_TIMEOUT, drains and exits normally.
 #include <cuda.h>
 
@@ -27,6 +39,13 @@
 namespace kmip {
 
 namespace {
+
+#ifndef KMIP_SWEEP_DEBUG
+#define KMIP_SWEEP_DEBUG 0
+#endif
+// Timing experiments (skip parts of the selection, per-role cycle counters) exist only in debug
+// builds; in the normal build `dbg` folds to 0 and none of the checks below reach the hot loop.
+constexpr bool kSweepDebug = KMIP_SWEEP_DEBUG != 0;
 
 constexpr int BM = 128;  // query rows per tile = TMEM lanes
 constexpr int BN = 128;  // keys per tile = accumulator columns
@@ -62,23 +81,25 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                 ((uint32_t)(BM >> 4) << 24);
 
-template <int E, int NQT, int S>
+constexpr int ROOM = 32;  // pending candidate slots per row
+
+template <int KG, int NQT, int S>
 struct SmemPlan {
-    static constexpr int CAP = 32 * E;
-    static constexpr int ROW_STRIDE = CAP + 1;  // odd pitch: simultaneous appends hit distinct banks
-    static constexpr int NBARS = 3 + 2 * S + 4 * NQT;
+    static constexpr int LIST = 8 * KG;          // list slots per row (k <= LIST)
+    static constexpr int SLOTS = LIST + ROOM;    // cand_t per row
+    static constexpr int NBARS = 3 + 2 * S + 4;
 };
 
 struct Bars {
     uint32_t base;
-    int S, NQT;
+    int S;
     __device__ uint32_t q_full() const { return base; }
     __device__ uint32_t q_empty() const { return base + 8; }
     __device__ uint32_t done() const { return base + 16; }
     __device__ uint32_t k_full(int s) const { return base + 8 * (3 + s); }
     __device__ uint32_t k_empty(int s) const { return base + 8 * (3 + S + s); }
-    __device__ uint32_t t_full(int qt, int b) const { return base + 8 * (3 + 2 * S + qt * 2 + b); }
-    __device__ uint32_t t_empty(int qt, int b) const { return base + 8 * (3 + 2 * S + 2 * NQT + qt * 2 + b); }
+    __device__ uint32_t t_full(int b) const { return base + 8 * (3 + 2 * S + b); }
+    __device__ uint32_t t_empty(int b) const { return base + 8 * (3 + 2 * S + 2 + b); }
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -88,68 +109,127 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     return false;
 }
 
-// Threshold test and candidate append for 32 consecutive scores of this thread's row.
-// Warp-uniform control flow: the rescan and the compactions are entered by all 32 lanes.
-template <int E>
-__device__ __forceinline__ void filter_chunk(const uint32_t (&v)[32], int key0, int nvalid, float& tau, int& cnt,
-                                             cand_t* myrow, cand_t* wrows, int k, int lane) {
-    constexpr int CAP = 32 * E;
-    constexpr int RS = CAP + 1;
-    float f[32];
+// Per-row selection state of one thread.  The row's slots live in the warp's block of shared
+// memory in slot-major order (slot s of lane l at [s*32 + l]), so lock-step loops over slots are
+// bank-conflict free.  The k-entry list is unsorted; gmin caches the minimum of each 8-slot group
+// and lmin the minimum of the list (0 = an empty slot, so tau stays -inf until k real entries exist).
+template <int KG>
+struct RowSel {
+    cand_t gmin[KG];
+    cand_t lmin;
+    float tau;
+    int cnt;
+};
+
+template <int KG>
+__device__ __forceinline__ void row_init(RowSel<KG>& r, cand_t* wl, int k, int lane, bool rvalid) {
+#pragma unroll 1
+    for (int s = 0; s < 8 * KG; ++s) wl[s * 32 + lane] = (s < k) ? 0ull : ~0ull;  // slots past k are never the minimum
 #pragma unroll
-    for (int x = 0; x < 32; ++x) f[x] = __uint_as_float(v[x]);
-    if (nvalid < 32) {  // ragged end of the graph's key range: columns past it do not exist
+    for (int g = 0; g < KG; ++g) r.gmin[g] = (8 * g < k) ? 0ull : ~0ull;
+    r.lmin = 0ull;
+    r.tau = rvalid ? -CUDART_INF_F : CUDART_INF_F;
+    r.cnt = 0;
+}
+
+// All 32 lanes insert their pending candidates into their own lists, in lock step.
+template <int KG>
+__device__ __forceinline__ void flush_pending(RowSel<KG>& r, cand_t* wl, const cand_t* wp, int lane, bool rvalid) {
+    const int maxc = __reduce_max_sync(FULL, r.cnt);
+    __syncwarp();
+#pragma unroll 1
+    for (int t = 0; t < maxc; ++t) {
+        if (t < r.cnt) {
+            const uint2 raw = *reinterpret_cast<const uint2*>(wp + t * 32 + lane);  // {first key, fp32 bits}
+            const cand_t x = make_cand(__uint_as_float(raw.y), (int)raw.x);
+            if (x > r.lmin) {
+                int g = 0;
+                cand_t m = r.gmin[0];
 #pragma unroll
-        for (int x = 0; x < 32; ++x)
-            if (x >= nvalid) f[x] = -CUDART_INF_F;
-    }
-    float sub[4];
+                for (int q = 1; q < KG; ++q)
+                    if (r.gmin[q] < m) { m = r.gmin[q]; g = q; }
+                cand_t* grp = wl + (g * 8) * 32 + lane;
+                cand_t nm = x;
+                int pos = -1;
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        float m = ptx::max3(f[8 * g], f[8 * g + 1], f[8 * g + 2]);
-        m = ptx::max3(m, f[8 * g + 3], f[8 * g + 4]);
-        m = ptx::max3(m, f[8 * g + 5], f[8 * g + 6]);
-        sub[g] = fmaxf(m, f[8 * g + 7]);
-    }
-    const float gm = fmaxf(ptx::max3(sub[0], sub[1], sub[2]), sub[3]);
-    if (__any_sync(FULL, gm > tau)) {
-        const int room = CAP - k;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            if (__any_sync(FULL, sub[g] > tau)) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int x = 8 * g + c;
-                    if (f[x] > tau) {
-                        myrow[k + cnt] = make_cand(f[x], key0 + x);
-                        ++cnt;
-                    }
+                for (int s = 0; s < 8; ++s) {
+                    const cand_t y = grp[s * 32];
+                    if (y == m && pos < 0) pos = s; else nm = cmin(nm, y);
                 }
-                unsigned need = __ballot_sync(FULL, cnt > room - 8);
-                while (need) {
-                    const int r = __ffs(need) - 1;
-                    need &= need - 1;
-                    const int rc = __shfl_sync(FULL, cnt, r);
-                    const float nt = warp_compact_row<E>(wrows + r * RS, k, rc, lane);
-                    if (lane == r) {
-                        tau = nt;
-                        cnt = 0;
-                    }
-                }
+                grp[pos * 32] = x;
+#pragma unroll
+                for (int q = 0; q < KG; ++q)
+                    if (q == g) r.gmin[q] = nm;
+                cand_t lm = r.gmin[0];
+#pragma unroll
+                for (int q = 1; q < KG; ++q) lm = cmin(lm, r.gmin[q]);
+                r.lmin = lm;
+            }
+        }
+    }
+    r.cnt = 0;
+    if (rvalid) r.tau = r.lmin ? cand_score(r.lmin) : -CUDART_INF_F;
+}
+
+// Maxima of the eight 8-column groups of 64 consecutive columns (three-input max; all first-level
+// operations come before the second level so that they issue back to back), and of the two
+// 32-column quads.  RAGGED: columns at or past `nvalid` do not exist (end of the key range).
+template <bool RAGGED>
+__device__ __forceinline__ void half_maxima(uint32_t (&v)[64], int nvalid, float* sub, float* quad) {
+    if (RAGGED) {
+#pragma unroll
+        for (int x = 0; x < 64; ++x)
+            if (x >= nvalid) v[x] = 0xFF800000u;  // -inf
+    }
+    float m0[8], m1[8], m2[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const int o = 8 * g;
+        m0[g] = ptx::max3(__uint_as_float(v[o]), __uint_as_float(v[o + 1]), __uint_as_float(v[o + 2]));
+        m1[g] = ptx::max3(__uint_as_float(v[o + 3]), __uint_as_float(v[o + 4]), __uint_as_float(v[o + 5]));
+        m2[g] = fmaxf(__uint_as_float(v[o + 6]), __uint_as_float(v[o + 7]));
+    }
+#pragma unroll
+    for (int g = 0; g < 8; ++g) sub[g] = ptx::max3(m0[g], m1[g], m2[g]);
+    quad[0] = fmaxf(ptx::max3(sub[0], sub[1], sub[2]), sub[3]);
+    quad[1] = fmaxf(ptx::max3(sub[4], sub[5], sub[6]), sub[7]);
+}
+
+// Lists the groups of a row's tile that beat tau.  Lanes skip the 32-column quads whose maximum
+// does not beat it; inside a quad each group costs one predicated 8-byte store and one predicated
+// pointer bump.  A pending entry is {first key of the group, raw fp32 bits of the group maximum};
+// `pend` is the shared-memory byte address of the lane's next free slot (256 bytes apart).
+__device__ __forceinline__ void append_groups(const float (&sub)[16], const float (&quad)[4], float tau, int key_base,
+                                              uint32_t& pend) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        if (quad[c] > tau) {
+#pragma unroll
+            for (int g = 4 * c; g < 4 * c + 4; ++g) {
+                asm volatile(
+                    "{\n\t"
+                    ".reg .pred p;\n\t"
+                    "setp.gt.f32 p, %1, %2;\n\t"
+                    "@p st.shared.v2.b32 [%0], {%3, %1};\n\t"
+                    "@p add.u32 %0, %0, 256;\n\t"
+                    "}"
+                    : "+r"(pend)
+                    : "f"(sub[g]), "f"(tau), "r"(key_base + 8 * g)
+                    : "memory");
             }
         }
     }
 }
 
-template <int D, int E, int NQT, int S, bool DUMP>
-__global__ void __launch_bounds__(NQT * 128 + 64, 1)
+template <int D, int KG, int NQT, int S, bool DUMP>
+__global__ void __launch_bounds__(NQT * 128 + 96, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
-                       float* __restrict__ dump, int dump_ld) {
+                       float* __restrict__ dump, int dump_ld /* = N */, int dbg_arg, long long* __restrict__ timing) {
+    const int dbg = kSweepDebug ? dbg_arg : 0;
     using Sh = TcShape<D>;
-    using Sp = SmemPlan<E, NQT, S>;
-    constexpr int CAP = Sp::CAP, RS = Sp::ROW_STRIDE;
+    using Sp = SmemPlan<KG, NQT, S>;
     constexpr int NEPI = 4 * NQT;
     constexpr uint32_t TMEM_COLS = NQT * 2 * BN;
 
@@ -158,26 +238,25 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     uint8_t* sQ = smem;
     uint8_t* sK = sQ + NQT * Sh::TILE_BYTES;
     cand_t* sRows = reinterpret_cast<cand_t*>(sK + S * Sh::TILE_BYTES);
-    uint64_t* sBars = reinterpret_cast<uint64_t*>(sRows + NQT * 128 * RS);
+    uint64_t* sBars = reinterpret_cast<uint64_t*>(sRows + NQT * 128 * Sp::SLOTS);
     uint32_t* sTmem = reinterpret_cast<uint32_t*>(sBars + Sp::NBARS);
     volatile int* sAbort = reinterpret_cast<volatile int*>(sTmem + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    Bars bars{ptx::smem_u32(sBars), S, NQT};
+    Bars bars{ptx::smem_u32(sBars), S};
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bars.q_full(), 1);
-        ptx::mbar_init(bars.q_empty(), 1);
-        ptx::mbar_init(bars.done(), 1);
+        ptx::mbar_init(bars.q_empty(), 2);  // both MMA issuers commit to it
+        ptx::mbar_init(bars.done(), 2);
         for (int s = 0; s < S; ++s) {
             ptx::mbar_init(bars.k_full(s), 1);
             ptx::mbar_init(bars.k_empty(s), 1);
         }
-        for (int qt = 0; qt < NQT; ++qt)
-            for (int b = 0; b < 2; ++b) {
-                ptx::mbar_init(bars.t_full(qt, b), 1);
-                ptx::mbar_init(bars.t_empty(qt, b), 4);  // one arrival per selection warp of the tile
-            }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(bars.t_full(b), 1);
+            ptx::mbar_init(bars.t_empty(b), NEPI);  // one arrival per selection warp
+        }
         *sAbort = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
@@ -219,41 +298,48 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     ptx::mbar_arrive_expect_tx(bars.k_full(s), Sh::TILE_BYTES);
                     for (int ch = 0; ch < Sh::KCH; ++ch)
                         ptx::tma_load_2d(ptx::smem_u32(sK + s * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmK,
-                                         h * D + ch * 64, it.key_lo + j * BN, bars.k_full(s));
+                                         ch * 64, h * dump_ld + it.key_lo + j * BN, bars.k_full(s));
                 }
                 ++ic;
             }
             if (!ok) {
                 // give copies that are still in flight a bounded time to land before the CTA exits
-                const uint64_t t0 = ptx::globaltimer_ns();
+                const long long t0 = clock64();
                 for (int s = 0; s < S && kt > 0; ++s) {
                     const int last = kt - 1 - ((kt - 1 - s) % S + S) % S;  // last tile issued into stage s
                     if (last < 0) continue;
-                    while (!ptx::mbar_try_wait(bars.k_full(s), (last / S) & 1) &&
-                           ptx::globaltimer_ns() - t0 < 20000000ull) {}
+                    while (!ptx::mbar_try_wait(bars.k_full(s), (last / S) & 1) && clock64() - t0 < 40000000ll) {}
                 }
             }
         }
-    } else if (warp == NEPI + 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == NEPI + 1 || warp == NEPI + 2) {
+        // ------------------------------------------------------------------ MMA issuers
+        // Two threads in two warps: issuer p takes the key tiles with running number kt = p (mod 2),
+        // i.e. accumulator buffer p, so the barrier waits and the commit of one overlap with the
+        // MMAs of the other.  Per tile an issuer runs the MMAs of every query tile and commits
+        // once; the commit tells the selection warps that the scores are ready and (forwarded by
+        // selection warp 0) that the key stage can be refilled.
         if (lane == 0) {
+            const int mine = warp - (NEPI + 1);
             int kt = 0, ic = 0;
-            int tc[2] = {0, 0};
             bool ok = true;
+            long long w_kfull = 0, w_tempty = 0, t_begin = clock64();
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem it = items[w % n_items];
                 const int nq = (NQT == 2 && it.nrows > BM) ? 2 : 1;
                 if (!(ok = wait_or_abort(bars.q_full(), ic & 1, sAbort, sb, 3))) break;
                 ptx::tc_fence_after();
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
-                for (int j = 0; ok && j < ntiles; ++j, ++kt) {
-                    const int s = kt % S;
+                for (int j = 0; j < ntiles; ++j, ++kt) {
+                    const int s = kt % S, b = kt & 1;
+                    if (b != mine) continue;
+                    long long c0 = (dbg & 8) ? clock64() : 0;
                     if (!(ok = wait_or_abort(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4))) break;
+                    long long c1 = (dbg & 8) ? clock64() : 0;
+                    if (!(ok = wait_or_abort(bars.t_empty(b), ((kt >> 1) & 1) ^ 1, sAbort, sb, 5))) break;
+                    if (dbg & 8) { w_kfull += c1 - c0; w_tempty += clock64() - c1; }
                     ptx::tc_fence_after();
                     for (int qt = 0; qt < nq; ++qt) {
-                        const int b = tc[qt] & 1;
-                        if (!(ok = wait_or_abort(bars.t_empty(qt, b), ((tc[qt] >> 1) & 1) ^ 1, sAbort, sb, 5))) break;
-                        ptx::tc_fence_after();
                         const uint32_t d_tmem = tmem_base + (uint32_t)((qt * 2 + b) * BN);
 #pragma unroll
                         for (int ks = 0; ks < Sh::KSTEPS; ++ks) {
@@ -262,88 +348,136 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                             const uint64_t db = make_smem_desc<D>(ptx::smem_u32(sK + s * Sh::TILE_BYTES + off));
                             ptx::mma_bf16_ss(d_tmem, da, db, kInstrDesc, ks > 0 ? 1u : 0u);
                         }
-                        ptx::mma_commit(bars.t_full(qt, b));
-                        ++tc[qt];
                     }
-                    if (!ok) break;
-                    ptx::mma_commit(bars.k_empty(s));
+                    ptx::mma_commit(bars.t_full(b));
                 }
                 if (!ok) break;
                 ptx::mma_commit(bars.q_empty());
                 ++ic;
             }
+            if ((dbg & 8) && timing && mine == 0) {
+                timing[blockIdx.x * 8 + 0] = clock64() - t_begin;
+                timing[blockIdx.x * 8 + 1] = w_kfull;
+                timing[blockIdx.x * 8 + 2] = w_tempty;
+                timing[blockIdx.x * 8 + 3] = kt;
+            }
             // all issued MMAs must have retired before tensor memory is released
             ptx::mma_commit(bars.done());
-            const uint64_t t0 = ptx::globaltimer_ns();
-            while (!ptx::mbar_try_wait(bars.done(), 0) && ptx::globaltimer_ns() - t0 < 1000000000ull) {}
+            const long long t0 = clock64();
+            while (!ptx::mbar_try_wait(bars.done(), 0) && clock64() - t0 < 2000000000ll) {}
         }
-    } else {
+    } else if (warp < NEPI) {
         // ------------------------------------------------------------------ selection warps
         const int qt = warp >> 2, quarter = warp & 3;
-        cand_t* wrows = sRows + (qt * 128 + quarter * 32) * RS;
-        cand_t* myrow = wrows + lane * RS;
+        cand_t* wl = sRows + (size_t)(qt * 128 + quarter * 32) * Sp::SLOTS;  // this warp's block: list slots ...
+        cand_t* wp = wl + Sp::LIST * 32;                                     // ... then pending slots
+        const uint32_t wp_addr = ptx::smem_u32(wp + lane);                   // this lane's first pending slot
+        RowSel<KG> rs;
         int tcnt = 0;
         bool ok = true;
+        long long w_tfull = 0, t_work = 0, t_begin = clock64();
+        long long prof[4] = {0, 0, 0, 0};
         for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
             const int h = (int)(w / n_items);
             const WorkItem it = items[w % n_items];
-            if (qt * BM >= it.nrows) continue;  // this query tile is empty for the item
+            const bool active = qt * BM < it.nrows;  // an inactive query tile only keeps the barriers in step
             const int local = qt * BM + quarter * 32 + lane;
             const bool rvalid = local < it.nrows;
-            for (int t = 0; t < k; ++t) myrow[t] = 0ull;
-            float tau = rvalid ? -CUDART_INF_F : CUDART_INF_F;
-            int cnt = 0;
+            if (active) row_init<KG>(rs, wl, k, lane, rvalid);
             __syncwarp();
             const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
             for (int j = 0; j < ntiles; ++j, ++tcnt) {
                 const int b = tcnt & 1;
-                ok = wait_or_abort(bars.t_full(qt, b), (tcnt >> 1) & 1, sAbort, sb, 6);
+                const long long c0 = (dbg & 8) ? clock64() : 0;
+                ok = wait_or_abort(bars.t_full(b), (tcnt >> 1) & 1, sAbort, sb, 6);
                 ok = __all_sync(FULL, ok);
                 if (!ok) break;
+                const long long c1 = (dbg & 8) ? clock64() : 0;
+                // the tile's MMAs have retired, so its key stage can be refilled
+                if (warp == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((qt * 2 + b) * BN);
                 const int key0 = it.key_lo + j * BN;
                 const int ncol = min(BN, it.key_hi - key0);
-                uint32_t va[32], vb[32];
-                ptx::tmem_ld_32x32(taddr, va);
+                if (DUMP) {
+                    uint32_t v[BN];
+                    if (active) ptx::tmem_ld_32x128_sync(taddr, v);
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
+                    if (active && rvalid)
 #pragma unroll
-                for (int c = 0; c < BN / 32; c += 2) {
-                    ptx::tmem_ld_wait(va);
-                    ptx::tmem_ld_32x32(taddr + (c + 1) * 32, vb);
-                    if (DUMP) {
-                        if (rvalid)
-                            for (int x = 0; x < 32; ++x)
-                                if (c * 32 + x < ncol)
-                                    dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + c * 32 + x] = __uint_as_float(va[x]);
-                    } else {
-                        filter_chunk<E>(va, key0 + c * 32, ncol - c * 32, tau, cnt, myrow, wrows, k, lane);
+                        for (int x = 0; x < BN; ++x)
+                            if (x < ncol)
+                                dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + x] = __uint_as_float(v[x]);
+                } else {
+                    // two 64-column halves keep the register footprint small; the accumulator buffer
+                    // goes back to the MMA issuer as soon as the second half is in registers
+                    float sub[16], quad[4];
+                    uint32_t v[64];
+                    const bool ragged = ncol < BN;
+                    if (active) {
+                        ptx::tmem_ld_32x64_sync(taddr, v);
+                        if (!(dbg & 2)) {
+                            if (ragged) half_maxima<true>(v, ncol, sub, quad);
+                            else half_maxima<false>(v, ncol, sub, quad);
+                        }
+                        ptx::tmem_ld_32x64_sync(taddr + 64, v);
                     }
-                    ptx::tmem_ld_wait(vb);
-                    if (c + 2 < BN / 32) ptx::tmem_ld_32x32(taddr + (c + 2) * 32, va);
-                    if (DUMP) {
-                        if (rvalid)
-                            for (int x = 0; x < 32; ++x)
-                                if ((c + 1) * 32 + x < ncol)
-                                    dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + (c + 1) * 32 + x] = __uint_as_float(vb[x]);
-                    } else {
-                        filter_chunk<E>(vb, key0 + (c + 1) * 32, ncol - (c + 1) * 32, tau, cnt, myrow, wrows, k, lane);
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
+                    if (active && !(dbg & 2)) {
+                        if (ragged) half_maxima<true>(v, ncol - 64, sub + 8, quad + 2);
+                        else half_maxima<false>(v, ncol - 64, sub + 8, quad + 2);
+                        const float gm = fmaxf(fmaxf(quad[0], quad[1]), fmaxf(quad[2], quad[3]));
+                        if (!(dbg & 1)) {
+                            const long long p0 = (dbg & 8) ? clock64() : 0;
+                            if (gm > rs.tau) {  // only lanes with a hit list their groups
+                                uint32_t pend = wp_addr + (uint32_t)rs.cnt * 256u;
+                                append_groups(sub, quad, rs.tau, key0, pend);
+                                rs.cnt = (int)((pend - wp_addr) >> 8);
+                            }
+                            const bool need = __any_sync(FULL, rs.cnt > ROOM - 16);  // a tile adds at most 16 groups per row
+                            if (dbg & 8) { prof[0] += clock64() - p0; prof[1] += __any_sync(FULL, gm > rs.tau) ? 1 : 0; }
+                            if (need) {
+                                const long long p1 = (dbg & 8) ? clock64() : 0;
+                                flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                                if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
+                            }
+                        } else if (gm == 123.456f) {
+                            rs.tau = 0.0f;  // timing experiment: keep the maxima alive
+                        }
+                    } else if (active && v[0] == 0x12345678u && v[63] == 1u) {
+                        rs.tau = 0.0f;  // timing experiment: keep the loads alive
                     }
                 }
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bars.t_empty(qt, b));
+                if (dbg & 8) { w_tfull += c1 - c0; t_work += clock64() - c1; }
             }
             if (!ok) break;
-            if (!DUMP) {
-                // finalise: one last compaction per row leaves the sorted best k in slots [0,k)
+            if (!DUMP && active) {
+                // finalise: drain the pending slots, then store each row's k groups (first key and
+                // group maximum, unsorted; empty slots as -1 / -inf) for the rescoring kernel
+                flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                __syncwarp();
                 const int nloc = min(32, it.nrows - (qt * BM + quarter * 32));
                 for (int r = 0; r < nloc; ++r) {
-                    const int rc = __shfl_sync(FULL, cnt, r);
-                    warp_compact_row<E>(wrows + r * RS, k, rc, lane);
                     const size_t o = ((size_t)(it.row0 + qt * BM + quarter * 32 + r) * H + h) * k;
-                    warp_store_row(wrows + r * RS, k, lane, topk_idx + o, topk_score + o);
+                    for (int t = lane; t < k; t += 32) {
+                        const cand_t c = wl[t * 32 + r];
+                        topk_idx[o + t] = c ? cand_index(c) : -1;
+                        topk_score[o + t] = c ? cand_score(c) : -CUDART_INF_F;
+                    }
                 }
+                __syncwarp();
             }
+        }
+        if ((dbg & 8) && timing && threadIdx.x == 0) {
+            timing[blockIdx.x * 8 + 4] = clock64() - t_begin;
+            timing[blockIdx.x * 8 + 5] = w_tfull;
+            timing[blockIdx.x * 8 + 6] = t_work;
+            timing[blockIdx.x * 8 + 7] = tcnt;
+            for (int i = 0; i < 4; ++i) timing[148 * 8 + blockIdx.x * 8 + i] = prof[i];
         }
     }
 
@@ -356,6 +490,9 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 }
 
 // ------------------------------------------------------------------------------------------- host
+int g_debug_flags = 0;  // timing experiments only (see set_score_select_debug_flags)
+long long* g_debug_timing = nullptr;  // device buffer [grid][8] of cycle counters when flag bit 3 is set
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -372,14 +509,16 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// Tensor map over one [N, H*d] bf16 array; a box is 128 rows x one swizzle span of columns.
+// Tensor map over a bf16 matrix of `rows` rows of `row_elems` elements; a box is 128 rows x one
+// swizzle span of columns.  Q is [N, H*d] (a head is a column block); the regrouped keys are
+// [H*N, d] (a head is a row block, so a key tile is one contiguous piece of memory).
 template <int D>
-bool make_tensor_map(CUtensorMap* tm, const void* base, int64_t N, int H) {
+bool make_tensor_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t row_elems) {
     using Sh = TcShape<D>;
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
-    const cuuint64_t gdim[2] = {(cuuint64_t)H * D, (cuuint64_t)N};
-    const cuuint64_t gstride[1] = {(cuuint64_t)H * D * 2};
+    const cuuint64_t gdim[2] = {(cuuint64_t)row_elems, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)row_elems * 2};
     const cuuint32_t box[2] = {(cuuint32_t)Sh::BOX_INNER, 128u};
     const cuuint32_t estr[2] = {1u, 1u};
     const CUtensorMapSwizzle sw = Sh::SWB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
@@ -401,37 +540,42 @@ int sm_count() {
     return sms[dev];
 }
 
-template <int D, int E, int NQT, int S, bool DUMP>
+template <int D, int KG, int NQT, int S, bool DUMP>
 cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     using Sh = TcShape<D>;
-    using Sp = SmemPlan<E, NQT, S>;
-    constexpr size_t smem_bytes = 1024 + (size_t)(NQT + S) * Sh::TILE_BYTES + (size_t)NQT * 128 * Sp::ROW_STRIDE * 8 +
-                                  (size_t)Sp::NBARS * 8 + 16;
+    using Sp = SmemPlan<KG, NQT, S>;
+    constexpr size_t smem_bytes = 1024 + (size_t)(NQT + S) * Sh::TILE_BYTES + (size_t)NQT * 128 * Sp::SLOTS * 8 +
+                                  (size_t)Sp::NBARS * 8 + 16 + 64;
     static_assert(smem_bytes <= 232448, "shared memory budget of one CTA");
     CUtensorMap tmQ, tmK;
-    if (!make_tensor_map<D>(&tmQ, a.Q, a.N, a.H) || !make_tensor_map<D>(&tmK, a.K, a.N, a.H))
+    if (!make_tensor_map<D>(&tmQ, a.Q, a.N, (int64_t)a.H * D) ||
+        !make_tensor_map<D>(&tmK, a.ws + w.kpack_off, a.N * a.H, D))
         return cudaErrorInvalidValue;
-    auto kern = score_select_tc_kernel<D, E, NQT, S, DUMP>;
+    auto kern = score_select_tc_kernel<D, KG, NQT, S, DUMP>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (err != cudaSuccess) return err;
     const long long max_total = (long long)w.max_items * a.H;
     const int grid = (int)std::min<long long>(sm_count(), max_total);
-    kern<<<grid, NQT * 128 + 64, smem_bytes, a.stream>>>(
+    kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
-        a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N);
+        a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing);
     return cudaGetLastError();
 }
 
 template <int D, bool DUMP>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
-    constexpr int S = D <= 32 ? 4 : 3;
-    if constexpr (D <= 64) {
-        if (a.k <= 32) return launch_cfg<D, 2, 2, S, DUMP>(a, w, dump);
-        return launch_cfg<D, 4, 1, S, DUMP>(a, w, dump);
-    } else {
-        if (a.k <= 32) return launch_cfg<D, 2, 1, S, DUMP>(a, w, dump);
-        return cudaErrorNotSupported;
+    // (list groups KG, query tiles per CTA, key stages) by k and head width; shared memory decides
+    if (a.k <= 32) {
+        if constexpr (D <= 32) return launch_cfg<D, 4, 2, 6, DUMP>(a, w, dump);
+        else if constexpr (D == 64) return launch_cfg<D, 4, 2, 3, DUMP>(a, w, dump);
+        else return launch_cfg<D, 4, 1, 3, DUMP>(a, w, dump);
     }
+    if (a.k <= 64) {
+        if constexpr (D <= 64) return launch_cfg<D, 8, 1, 4, DUMP>(a, w, dump);
+        else return launch_cfg<D, 8, 1, 3, DUMP>(a, w, dump);
+    }
+    if constexpr (D <= 64) return launch_cfg<D, 16, 1, 3, DUMP>(a, w, dump);
+    else return cudaErrorNotSupported;
 }
 
 template <bool DUMP>
@@ -447,13 +591,18 @@ cudaError_t launch_any(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
 
 }  // namespace
 
+// bit 0: skip the candidate path, bit 1: skip the whole filter.  Results are then meaningless;
+// used only to time the tensor pipeline and the tensor-memory loads in isolation.
+void set_score_select_debug_flags(int flags) { g_debug_flags = flags; }
+void set_score_select_debug_timing(long long* buf) { g_debug_timing = buf; }
+
 bool score_select_tc_supported(int32_t d, int32_t k) {
     if (d != 16 && d != 32 && d != 64 && d != 128) return false;
-    if (k <= 32) return true;
-    return k <= 96 && d <= 64;
+    if (k <= 64) return true;
+    return k <= 128 && d <= 64;
 }
 
-int score_select_tc_rows_per_item(int32_t d, int32_t k) { return (k <= 32 && d <= 64) ? 256 : 128; }
+int score_select_tc_rows_per_item(int32_t d, int32_t k) { return (k <= 32 && d <= 64) ? 256 : 128; }  // 128 * query tiles per CTA
 
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w) {
     return launch_any<false>(a, w, nullptr);

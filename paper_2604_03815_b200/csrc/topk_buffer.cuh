@@ -23,7 +23,7 @@ typedef unsigned long long cand_t;
 
 __device__ __forceinline__ uint32_t order_bits(float s) {
     const uint32_t u = __float_as_uint(s);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);  // negative: flip all bits; else set the sign bit
 }
 __device__ __forceinline__ float unorder_bits(uint32_t u) {
     return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
@@ -94,6 +94,38 @@ __device__ __forceinline__ float warp_compact_row(cand_t* row, int k, int cnt, i
     __syncwarp();
     const cand_t kth = row[k - 1];
     return kth ? cand_score(kth) : -CUDART_INF_F;
+}
+
+// Same result as warp_compact_row for k <= 32 and cnt <= 32, with less work: the kept list
+// (one key per lane, already sorted) is merged with the sorted pending keys instead of sorting
+// all slots again.  max(list[i], pending[31-i]) holds the 32 largest of both and is bitonic, so
+// five more compare-exchange stages sort it.
+__device__ __forceinline__ float warp_merge_row32(cand_t* row, int k, int cnt, int lane) {
+    __syncwarp();
+    cand_t lst = (lane < k) ? row[lane] : 0ull;
+    cand_t pend[1] = {(lane < cnt) ? row[k + lane] : 0ull};
+    warp_sort_desc<1>(pend, lane);
+    const cand_t rev = __shfl_sync(0xFFFFFFFFu, pend[0], 31 - lane);
+    cand_t m = cmax(lst, rev);
+#pragma unroll
+    for (int j = 16; j > 0; j >>= 1) {
+        const cand_t o = __shfl_xor_sync(0xFFFFFFFFu, m, j);
+        m = ((lane & j) == 0) ? cmax(m, o) : cmin(m, o);
+    }
+    __syncwarp();
+    if (lane < k) row[lane] = m;
+    const cand_t kth = __shfl_sync(0xFFFFFFFFu, m, k - 1);
+    __syncwarp();
+    return kth ? cand_score(kth) : -CUDART_INF_F;
+}
+
+// Out-of-line entry points: compaction is rare, so one copy of its code is shared by all call
+// sites and stays out of the hot loop's instruction stream.
+template <int E>
+__device__ __noinline__ float compact_row_outlined(cand_t* row, int k, int cnt) {
+    const int lane = threadIdx.x & 31;
+    if (E == 2 && k <= 32 && cnt <= 32) return warp_merge_row32(row, k, cnt, lane);
+    return warp_compact_row<E>(row, k, cnt, lane);
 }
 
 // Write a finished row: slots [0,k) -> topk_idx / topk_score (empty slots: -1 / -inf).

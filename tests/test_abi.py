@@ -41,7 +41,8 @@ def test_version_and_status_strings(kb):
 def test_workspace_bytes_host_only(kb):
     f = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
     b = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
-    assert 256 < f < (1 << 20)
+    assert 500_000 * 4 * 32 * 2 < f < 500_000 * 4 * 32 * 2 + (1 << 20)   # K regrouped by head + work items
+    assert 256 < kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_FP32_EXACT, kb.PASS_FORWARD) < (1 << 20)
     pairs = 500_000 * 4 * 32
     assert 12 * pairs < b < 14 * pairs          # p, dS, pair list: 12 bytes per selected pair + O(N*H)
     for bad in [dict(d=24), dict(k=129), dict(mode=7)]:
