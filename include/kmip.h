@@ -124,9 +124,9 @@ int kmip_last_status(const void *workspace, void *stream, int *device_status);
  * to n forward and n backward calls (n <= 256) and makes the two passes record them around their
  * stages on the caller's stream; kmip_profile_enable(0) destroys them and turns recording off.
  * kmip_profile_read waits for the recorded events, adds up the stage times in milliseconds into
- * stage_ms[6] = {plan, score+select, softmax+gather-V, backward rows, inverse index, dK/dV
- * segments}, stores the number of forward / backward calls recorded in calls[2] and resets the
- * counters.  Process-wide state, not thread-safe, one device; leave it off on the hot path.
+ * stage_ms[7] = {plan (+ key regrouping), score+select sweep, rescoring of the candidate groups,
+ * softmax+gather-V, backward rows, inverse index, dK/dV segments}, stores the number of forward /
+ * backward calls recorded in calls[2] and resets the counters.  Process-wide state, not thread-safe, one device; leave it off on the hot path.
  */
 int kmip_profile_enable(int max_calls);
 int kmip_profile_read(double *stage_ms, int *calls);

@@ -121,7 +121,8 @@ def kmip_last_status(workspace, stream=None) -> int:
     return int(st.value)
 
 
-STAGES = ("plan", "score_select", "softmax_gather", "bwd_rows", "bwd_inverse_index", "bwd_segments")
+STAGES = ("plan", "score_select", "refine", "softmax_gather", "bwd_rows", "bwd_inverse_index", "bwd_segments")
+N_FWD_STAGES = 4
 
 
 def kmip_profile_enable(max_calls: int) -> None:
@@ -132,7 +133,7 @@ def kmip_profile_enable(max_calls: int) -> None:
 
 def kmip_profile_read():
     """Returns ({stage: total milliseconds}, forward calls, backward calls) since the last read."""
-    ms = (ctypes.c_double * 6)()
+    ms = (ctypes.c_double * 7)()
     calls = (ctypes.c_int * 2)()
     rc = lib().kmip_profile_read(ms, calls)
     if rc != KMIP_OK:

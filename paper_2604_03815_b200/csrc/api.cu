@@ -24,7 +24,7 @@ struct Profile {
     bool on = false;
     int max_calls = 0;
     int n_fwd = 0, n_bwd = 0;
-    cudaEvent_t fwd[kProfMaxCalls][4];
+    cudaEvent_t fwd[kProfMaxCalls][5];
     cudaEvent_t bwd[kProfMaxCalls][4];
 };
 Profile g_prof;
@@ -83,12 +83,12 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     if (tc && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 256) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
-    cudaError_t e1 = tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a);
-    if (e1 == cudaSuccess && tc) e1 = launch_refine_topk(a);
-    if (e1 != cudaSuccess) return KMIP_ERR_CUDA;
+    if ((tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], a.stream);
-    if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (tc && launch_refine_topk(a) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[3], a.stream);
+    if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (ev) cudaEventRecord(ev[4], a.stream);
     return KMIP_OK;
 }
 
@@ -127,18 +127,22 @@ int kmip_last_status(const void* workspace, void* stream, int* device_status) {
 
 int kmip_profile_enable(int max_calls) {
     if (g_prof.on) {
-        for (int i = 0; i < g_prof.max_calls; ++i)
-            for (int e = 0; e < 4; ++e) { cudaEventDestroy(g_prof.fwd[i][e]); cudaEventDestroy(g_prof.bwd[i][e]); }
+        for (int i = 0; i < g_prof.max_calls; ++i) {
+            for (int e = 0; e < 5; ++e) cudaEventDestroy(g_prof.fwd[i][e]);
+            for (int e = 0; e < 4; ++e) cudaEventDestroy(g_prof.bwd[i][e]);
+        }
         g_prof.on = false;
     }
     g_prof.n_fwd = g_prof.n_bwd = 0;
     g_prof.max_calls = 0;
     if (max_calls <= 0) return KMIP_OK;
     if (max_calls > kProfMaxCalls) max_calls = kProfMaxCalls;
-    for (int i = 0; i < max_calls; ++i)
+    for (int i = 0; i < max_calls; ++i) {
+        for (int e = 0; e < 5; ++e)
+            if (cudaEventCreate(&g_prof.fwd[i][e]) != cudaSuccess) return KMIP_ERR_CUDA;
         for (int e = 0; e < 4; ++e)
-            if (cudaEventCreate(&g_prof.fwd[i][e]) != cudaSuccess || cudaEventCreate(&g_prof.bwd[i][e]) != cudaSuccess)
-                return KMIP_ERR_CUDA;
+            if (cudaEventCreate(&g_prof.bwd[i][e]) != cudaSuccess) return KMIP_ERR_CUDA;
+    }
     g_prof.max_calls = max_calls;
     g_prof.on = true;
     return KMIP_OK;
@@ -146,19 +150,20 @@ int kmip_profile_enable(int max_calls) {
 
 int kmip_profile_read(double* stage_ms, int* calls) {
     if (!stage_ms || !calls) return KMIP_ERR_INVALID_ARG;
-    for (int s = 0; s < 6; ++s) stage_ms[s] = 0.0;
+    for (int s = 0; s < 7; ++s) stage_ms[s] = 0.0;
     calls[0] = g_prof.n_fwd;
     calls[1] = g_prof.n_bwd;
     if (!g_prof.on) return KMIP_OK;
     for (int pass = 0; pass < 2; ++pass) {
         const int n = pass ? g_prof.n_bwd : g_prof.n_fwd;
+        const int n_stage = pass ? 3 : 4;
         for (int i = 0; i < n; ++i) {
             cudaEvent_t* ev = pass ? g_prof.bwd[i] : g_prof.fwd[i];
-            if (cudaEventSynchronize(ev[3]) != cudaSuccess) return KMIP_ERR_CUDA;
-            for (int s = 0; s < 3; ++s) {
+            if (cudaEventSynchronize(ev[n_stage]) != cudaSuccess) return KMIP_ERR_CUDA;
+            for (int s = 0; s < n_stage; ++s) {
                 float ms = 0.0f;
                 if (cudaEventElapsedTime(&ms, ev[s], ev[s + 1]) != cudaSuccess) return KMIP_ERR_CUDA;
-                stage_ms[pass * 3 + s] += ms;
+                stage_ms[pass * 4 + s] += ms;
             }
         }
     }
