@@ -119,8 +119,9 @@ cudaError_t launch_d(const FwdArgs& a) {
     refine_topk_kernel<T, D, E_><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
         static_cast<const T*>(a.Q), static_cast<const T*>(a.K), a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
         a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws))
-    if (a.k <= 32) KMIP_LAUNCH_REFINE(2);
-    else if (a.k <= 96) KMIP_LAUNCH_REFINE(4);
+    // pending room CAP-k >= 96, so that the survivors of a row (rarely more than 2k) fit without
+    // intermediate compactions
+    if (a.k <= 32) KMIP_LAUNCH_REFINE(4);
     else KMIP_LAUNCH_REFINE(8);
 #undef KMIP_LAUNCH_REFINE
     return cudaGetLastError();
