@@ -42,7 +42,8 @@ typedef enum {
     KMIP_ERR_WORKSPACE = 3,    /* workspace smaller than kmip_attn_workspace_bytes reports */
     KMIP_ERR_CUDA = 4,         /* a CUDA runtime call or a kernel launch failed */
     KMIP_ERR_TIMEOUT = 5,      /* device side: a bounded wait inside a kernel ran out */
-    KMIP_ERR_BAD_OFFSETS = 6   /* device side: graph_offsets is not a valid CSR row-pointer array */
+    KMIP_ERR_BAD_OFFSETS = 6,  /* device side: graph_offsets is not a valid CSR row-pointer array */
+    KMIP_ERR_TOO_LARGE = 7     /* kmip_attn_forward_static_scratch: the problem needs more than the built-in scratch */
 } kmip_status_t;
 
 typedef enum {
@@ -109,6 +110,41 @@ int kmip_attn_backward(const void *Q, const void *K, const void *V,
                        const int32_t *topk_idx, const float *topk_score,
                        void *dQ, void *dK, void *dV,
                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Size in bytes of the scratch array that is built into the library for
+ * kmip_attn_forward_static_scratch (8 MiB; each GPU that loads the library holds it until the
+ * process exits).
+ */
+#define KMIP_STATIC_SCRATCH_BYTES ((size_t)8 << 20)
+
+/*
+ * The forward pass of kmip_attn_forward for callers that cannot provide a workspace because they
+ * are not allowed to allocate device memory - for example a plug-in inside a framework that owns
+ * all device memory, or a serving loop whose memory pool is frozen after start-up (an allocation
+ * would also synchronise the device).  The paper has no counterpart; this is packaging only.
+ * Same arguments, results and status codes as kmip_attn_forward, except:
+ *   - there is no workspace argument: the scratch is a fixed KMIP_STATIC_SCRATCH_BYTES array inside
+ *     the library.  A problem whose kmip_attn_workspace_bytes(..., KMIP_PASS_FORWARD) exceeds it is
+ *     refused with KMIP_ERR_TOO_LARGE before anything is enqueued.  In tensor-core mode the scratch
+ *     is dominated by one bf16 copy of K, so the limit is about N*H*d <= 4.1 million elements
+ *     (e.g. 32 000 nodes at H = 4, d = 32); fp32 mode needs 16 bytes per 128 nodes and per graph.
+ *   - device_status (DEVICE pointer, may be NULL): if given, the device status word of this call
+ *     (KMIP_OK, KMIP_ERR_TIMEOUT or KMIP_ERR_BAD_OFFSETS) is copied there on `stream` after the
+ *     kernels, since there is no workspace for kmip_last_status to read.
+ *   - the call itself calls no cudaMalloc / cudaFree or any other allocating routine.  The first call
+ *     on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - every call on a device uses the same array: two calls whose kernels can overlap on the GPU
+ *     (different streams, or several host threads) race and give undefined results; calls on one
+ *     stream are safe back to back.  The array keeps the last call's contents; each call clears or
+ *     rewrites every part it reads.
+ */
+int kmip_attn_forward_static_scratch(const void *Q, const void *K, const void *V,
+                                     const int32_t *graph_offsets, int32_t G, int64_t N,
+                                     int32_t H, int32_t d, int32_t k, int mode,
+                                     void *out, int32_t *topk_idx, float *topk_score,
+                                     int32_t *device_status, void *stream);
 
 /*
  * Synchronises `stream`, then copies the device status word of the last call that used

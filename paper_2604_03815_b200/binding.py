@@ -18,6 +18,7 @@ KMIP_ERR_WORKSPACE = 3
 KMIP_ERR_CUDA = 4
 KMIP_ERR_TIMEOUT = 5
 KMIP_ERR_BAD_OFFSETS = 6
+KMIP_ERR_TOO_LARGE = 7
 KMIP_BF16_TC = 0
 KMIP_FP32_EXACT = 1
 PASS_FORWARD = 0
@@ -55,6 +56,8 @@ def lib() -> ctypes.CDLL:
                                          P, P, P, P, sz, P]
         L.kmip_last_status.restype = ctypes.c_int
         L.kmip_last_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_int)]
+        L.kmip_attn_forward_static_scratch.restype = ctypes.c_int
+        L.kmip_attn_forward_static_scratch.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, P, P, P, P, P]
         L.kmip_profile_enable.restype = ctypes.c_int
         L.kmip_profile_enable.argtypes = [ctypes.c_int]
         L.kmip_profile_read.restype = ctypes.c_int
@@ -98,6 +101,18 @@ def kmip_attn_forward(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score
                                        _ptr(out), _ptr(topk_idx), _ptr(topk_score), _ptr(workspace),
                                        0 if workspace is None else workspace.numel() * workspace.element_size(),
                                        _stream(stream)))
+
+
+def kmip_attn_forward_static_scratch(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score,
+                                     device_status=None, stream=None) -> int:
+    """Forward pass that uses the library's built-in scratch array instead of a caller workspace
+    (for callers that may not allocate device memory); returns the library's status code.
+    `device_status`, if given, is an int32 CUDA tensor that receives the device status word."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(lib().kmip_attn_forward_static_scratch(_ptr(Q), _ptr(K), _ptr(V), _ptr(graph_offsets), G, N, H, d, k,
+                                                      mode, _ptr(out), _ptr(topk_idx), _ptr(topk_score),
+                                                      _ptr(device_status), _stream(stream)))
 
 
 def kmip_attn_backward(Q, K, V, graph_offsets, k, mode, out, d_out, topk_idx, topk_score, dQ, dK, dV,

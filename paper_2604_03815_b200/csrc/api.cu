@@ -44,6 +44,7 @@ const char* kmip_status_string(int status) {
         case KMIP_ERR_CUDA: return "CUDA runtime or launch failure";
         case KMIP_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case KMIP_ERR_BAD_OFFSETS: return "graph_offsets is not a valid CSR offset array";
+        case KMIP_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in array holds";
         default: return "unknown status";
     }
 }
