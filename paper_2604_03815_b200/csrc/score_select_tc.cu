@@ -195,15 +195,16 @@ __device__ __forceinline__ void half_maxima(uint32_t (&v)[64], int nvalid, float
     quad[1] = fmaxf(ptx::max3(sub[4], sub[5], sub[6]), sub[7]);
 }
 
-// Lists the groups of a row's tile that beat tau.  Lanes skip the 32-column quads whose maximum
-// does not beat it; inside a quad each group costs one predicated 8-byte store and one predicated
-// pointer bump.  A pending entry is {first key of the group, raw fp32 bits of the group maximum};
-// `pend` is the shared-memory byte address of the lane's next free slot (256 bytes apart).
+// Lists the groups of a row's tile that beat tau.  Control flow is warp-uniform: a 32-column quad is
+// visited when any lane has a hit in it (one vote), and inside a quad each group costs one compare,
+// one predicated 8-byte store and one predicated pointer bump.  A pending entry is {first key of
+// the group, raw fp32 bits of the group maximum}; `pend` is the shared-memory byte address of the
+// lane's next free slot (256 bytes apart).
 __device__ __forceinline__ void append_groups(const float (&sub)[16], const float (&quad)[4], float tau, int key_base,
                                               uint32_t& pend) {
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        if (quad[c] > tau) {
+        if (__any_sync(FULL, quad[c] > tau)) {
 #pragma unroll
             for (int g = 4 * c; g < 4 * c + 4; ++g) {
                 asm volatile(
@@ -433,17 +434,16 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         const float gm = fmaxf(fmaxf(quad[0], quad[1]), fmaxf(quad[2], quad[3]));
                         if (!(dbg & 1)) {
                             const long long p0 = (dbg & 8) ? clock64() : 0;
-                            if (gm > rs.tau) {  // only lanes with a hit list their groups
+                            if (__any_sync(FULL, gm > rs.tau)) {  // some lane of the warp has a hit in this tile
                                 uint32_t pend = wp_addr + (uint32_t)rs.cnt * 256u;
                                 append_groups(sub, quad, rs.tau, key0, pend);
                                 rs.cnt = (int)((pend - wp_addr) >> 8);
-                            }
-                            const bool need = __any_sync(FULL, rs.cnt > ROOM - 16);  // a tile adds at most 16 groups per row
-                            if (dbg & 8) { prof[0] += clock64() - p0; prof[1] += __any_sync(FULL, gm > rs.tau) ? 1 : 0; }
-                            if (need) {
-                                const long long p1 = (dbg & 8) ? clock64() : 0;
-                                flush_pending<KG>(rs, wl, wp, lane, rvalid);
-                                if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
+                                if (dbg & 8) { prof[0] += clock64() - p0; ++prof[1]; }
+                                if (__any_sync(FULL, rs.cnt > ROOM - 16)) {  // a tile adds at most 16 groups per row
+                                    const long long p1 = (dbg & 8) ? clock64() : 0;
+                                    flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                                    if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
+                                }
                             }
                         } else if (gm == 123.456f) {
                             rs.tau = 0.0f;  // timing experiment: keep the maxima alive
