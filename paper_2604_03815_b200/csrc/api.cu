@@ -176,6 +176,11 @@ int kmip_profile_read(double* stage_ms, int* calls) {
 void kmip_debug_set_flags(int flags) { set_score_select_debug_flags(flags); }
 void kmip_debug_set_timing(void* buf) { set_score_select_debug_timing(static_cast<long long*>(buf)); }
 
+// ---- test hook (not part of kmip.h): makes one bounded device-side wait run out, see score_select_tc.cu
+void kmip_debug_fault_test(int drop_first_tile, long long wait_limit_cycles) {
+    set_score_select_fault_test(drop_first_tile, wait_limit_cycles);
+}
+
 // ---- test hook (not part of kmip.h): dense scores of the tensor-core pipeline -----------------
 // Writes S[h][i][j] = q_i^h . k_j^h (fp32, [H, N, N]) for ONE graph of N <= 8192 nodes through the
 // same TMA / tcgen05 path as the forward pass, so tests can check the contraction element-wise.

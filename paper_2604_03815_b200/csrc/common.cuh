@@ -170,6 +170,7 @@ bool score_select_tc_supported(int32_t d, int32_t k);
 int score_select_tc_rows_per_item(int32_t d, int32_t k);
 void set_score_select_debug_flags(int flags);
 void set_score_select_debug_timing(long long* buf);
+void set_score_select_fault_test(int drop_first_tile, long long wait_limit_cycles);
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump);
 // refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k

@@ -103,8 +103,8 @@ struct Bars {
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                              StatusBlock* sb, int who) {
-    if (ptx::mbar_wait_bounded(bar, parity, abort_flag)) return true;
+                                              StatusBlock* sb, int who, long long limit) {
+    if (ptx::mbar_wait_bounded(bar, parity, abort_flag, limit)) return true;
     record_status(sb, KMIP_ERR_TIMEOUT, who);
     return false;
 }
@@ -227,7 +227,8 @@ __global__ void __launch_bounds__(NQT * 128 + 96, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
-                       float* __restrict__ dump, int dump_ld /* = N */, int dbg_arg, long long* __restrict__ timing) {
+                       float* __restrict__ dump, int dump_ld /* = N */, int dbg_arg, long long* __restrict__ timing,
+                       long long wait_limit, int drop_first_tile) {
     const int dbg = kSweepDebug ? dbg_arg : 0;
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
@@ -286,7 +287,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const int h = (int)(w / n_items);
                 const WorkItem it = items[w % n_items];
-                if (!(ok = wait_or_abort(bars.q_empty(), (ic & 1) ^ 1, sAbort, sb, 1))) break;
+                if (!(ok = wait_or_abort(bars.q_empty(), (ic & 1) ^ 1, sAbort, sb, 1, wait_limit))) break;
                 ptx::mbar_arrive_expect_tx(bars.q_full(), NQT * Sh::TILE_BYTES);
                 for (int qt = 0; qt < NQT; ++qt)
                     for (int ch = 0; ch < Sh::KCH; ++ch)
@@ -295,7 +296,10 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
                 for (int j = 0; j < ntiles; ++j, ++kt) {
                     const int s = kt % S;
-                    if (!(ok = wait_or_abort(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2))) break;
+                    if (!(ok = wait_or_abort(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit))) break;
+                    // failure-detection test hook: CTA 0 never loads its first key tile, so the waits on
+                    // that stage must run out, be reported and leave the context usable
+                    if (drop_first_tile && blockIdx.x == 0 && kt == 0) continue;
                     ptx::mbar_arrive_expect_tx(bars.k_full(s), Sh::TILE_BYTES);
                     for (int ch = 0; ch < Sh::KCH; ++ch)
                         ptx::tma_load_2d(ptx::smem_u32(sK + s * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmK,
@@ -328,16 +332,16 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem it = items[w % n_items];
                 const int nq = (NQT == 2 && it.nrows > BM) ? 2 : 1;
-                if (!(ok = wait_or_abort(bars.q_full(), ic & 1, sAbort, sb, 3))) break;
+                if (!(ok = wait_or_abort(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
                 ptx::tc_fence_after();
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
                 for (int j = 0; j < ntiles; ++j, ++kt) {
                     const int s = kt % S, b = kt & 1;
                     if (b != mine) continue;
                     long long c0 = (dbg & 8) ? clock64() : 0;
-                    if (!(ok = wait_or_abort(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4))) break;
+                    if (!(ok = wait_or_abort(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
                     long long c1 = (dbg & 8) ? clock64() : 0;
-                    if (!(ok = wait_or_abort(bars.t_empty(b), ((kt >> 1) & 1) ^ 1, sAbort, sb, 5))) break;
+                    if (!(ok = wait_or_abort(bars.t_empty(b), ((kt >> 1) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
                     if (dbg & 8) { w_kfull += c1 - c0; w_tempty += clock64() - c1; }
                     ptx::tc_fence_after();
                     for (int qt = 0; qt < nq; ++qt) {
@@ -390,7 +394,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             for (int j = 0; j < ntiles; ++j, ++tcnt) {
                 const int b = tcnt & 1;
                 const long long c0 = (dbg & 8) ? clock64() : 0;
-                ok = wait_or_abort(bars.t_full(b), (tcnt >> 1) & 1, sAbort, sb, 6);
+                ok = wait_or_abort(bars.t_full(b), (tcnt >> 1) & 1, sAbort, sb, 6, wait_limit);
                 ok = __all_sync(FULL, ok);
                 if (!ok) break;
                 const long long c1 = (dbg & 8) ? clock64() : 0;
@@ -491,7 +495,9 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
 // ------------------------------------------------------------------------------------------- host
 int g_debug_flags = 0;  // timing experiments only (see set_score_select_debug_flags)
-long long* g_debug_timing = nullptr;  // device buffer [grid][8] of cycle counters when flag bit 3 is set
+long long* g_debug_timing = nullptr;
+long long g_wait_limit_cycles = 8000000000ll;  // bound of every device-side wait, in SM clocks (about 4 s)
+int g_drop_first_tile = 0;                     // failure-detection test hook, see set_score_select_fault_test  // device buffer [grid][8] of cycle counters when flag bit 3 is set
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -558,7 +564,8 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     const int grid = (int)std::min<long long>(sm_count(), max_total);
     kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
-        a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing);
+        a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing, g_wait_limit_cycles,
+        g_drop_first_tile);
     return cudaGetLastError();
 }
 
@@ -595,6 +602,13 @@ cudaError_t launch_any(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
 // used only to time the tensor pipeline and the tensor-memory loads in isolation.
 void set_score_select_debug_flags(int flags) { g_debug_flags = flags; }
 void set_score_select_debug_timing(long long* buf) { g_debug_timing = buf; }
+
+// Test hook for the bounded waits: with drop_first_tile != 0 the next launches leave one key tile of
+// CTA 0 unloaded (a wait that nothing will ever satisfy); wait_limit_cycles <= 0 restores the default.
+void set_score_select_fault_test(int drop_first_tile, long long wait_limit_cycles) {
+    g_drop_first_tile = drop_first_tile;
+    g_wait_limit_cycles = wait_limit_cycles > 0 ? wait_limit_cycles : 8000000000ll;
+}
 
 bool score_select_tc_supported(int32_t d, int32_t k) {
     if (d != 16 && d != 32 && d != 64 && d != 128) return false;

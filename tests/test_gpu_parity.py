@@ -141,6 +141,28 @@ def test_bad_offsets_are_reported_by_the_device():
     pu.check_forward(w, pu.run_forward(w, (Q, K, V, dO, offs)))
 
 
+def test_bounded_wait_runs_out_and_is_reported():
+    """Failure detection without a GPU fault: a test hook leaves one key tile of CTA 0 unloaded, so the
+    waits on it can never be satisfied.  They must run out (limit shortened to ~0.2 s of SM clocks),
+    the kernel must return normally with KMIP_ERR_TIMEOUT in the status word, and the context must
+    stay usable for the next call."""
+    import ctypes
+    w = wl.iid_workload("s", 83, [2000], 1, 32, 8, wl.MODE_BF16_TC)
+    dev = pu.to_device(w)
+    Q, K, V, dO, offs = dev
+    L = kb.lib()
+    L.kmip_debug_fault_test.argtypes = [ctypes.c_int, ctypes.c_longlong]
+    b = kb.ForwardBuffers(w.N, 1, w.H, w.d, w.k, w.mode)
+    L.kmip_debug_fault_test(1, 400_000_000)
+    try:
+        assert kb.kmip_attn_forward(Q, K, V, offs, w.k, w.mode, b.out, b.topk_idx, b.topk_score, b.workspace) == kb.KMIP_OK
+        assert kb.kmip_last_status(b.workspace) == kb.KMIP_ERR_TIMEOUT
+    finally:
+        L.kmip_debug_fault_test(0, 0)
+    torch.cuda.synchronize()
+    pu.check_forward(w, pu.run_forward(w, dev))
+
+
 def test_workspace_too_small_is_refused():
     w = wl.iid_workload("s", 82, [300], 1, 32, 8, wl.MODE_BF16_TC)
     Q, K, V, dO, offs = pu.to_device(w)
