@@ -47,17 +47,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Same, but the hardware may keep the thread suspended for up to `hint_ns` while the phase is
+// incomplete (it resumes as soon as the phase completes), which keeps a waiting thread from
+// burning issue slots in a poll loop.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
 
-// Bounded wait: polls the barrier phase; gives up when `abort_flag` (shared memory) is set by
-// another thread or after roughly `limit_cycles` SM clocks (about 4 s by default), in which case
-// it sets the flag itself and returns false.  Callers leave their loops on false; nothing spins
-// forever.  The clock is read only every 1024 failed polls so the common case stays cheap.
+// Bounded wait: waits for the barrier phase in hardware-suspended slices of up to 20 us; gives up
+// when `abort_flag` (shared memory) is set by another thread or after roughly `limit_cycles` SM
+// clocks (about 4 s by default), in which case it sets the flag itself and returns false.
+// Callers leave their loops on false; nothing waits forever.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   long long limit_cycles = 8000000000ll) {
+    if (mbar_try_wait(bar, parity)) return true;
     uint32_t spins = 0;
     long long t0 = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 1023u) == 0u) {
+    while (!mbar_try_wait_suspend(bar, parity, 20000u)) {
+        if ((++spins & 15u) == 0u) {
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
