@@ -243,6 +243,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     uint64_t* sBars = reinterpret_cast<uint64_t*>(sRows + NQT * 128 * Sp::SLOTS);
     uint32_t* sTmem = reinterpret_cast<uint32_t*>(sBars + Sp::NBARS);
     volatile int* sAbort = reinterpret_cast<volatile int*>(sTmem + 1);
+    volatile int* sFlushReq = reinterpret_cast<volatile int*>(sTmem + 2);  // CTA-wide flush request counter
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     Bars bars{ptx::smem_u32(sBars), S};
@@ -260,6 +261,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ptx::mbar_init(bars.t_empty(b), NEPI);  // one arrival per selection warp
         }
         *sAbort = 0;
+        *sFlushReq = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -331,7 +333,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             long long w_kfull = 0, w_tempty = 0, t_begin = clock64();
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem it = items[w % n_items];
-                const int nq = (NQT == 2 && it.nrows > BM) ? 2 : 1;
+                const int nq = (NQT == 2 && it.nrows > BM && !(dbg & 16)) ? 2 : 1;  // dbg 16: timing experiment, one query tile only
                 if (!(ok = wait_or_abort(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
                 ptx::tc_fence_after();
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
@@ -378,14 +380,16 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         cand_t* wp = wl + Sp::LIST * 32;                                     // ... then pending slots
         const uint32_t wp_addr = ptx::smem_u32(wp + lane);                   // this lane's first pending slot
         RowSel<KG> rs;
+        int flush_seen = 0;
         int tcnt = 0;
         bool ok = true;
         long long w_tfull = 0, t_work = 0, t_begin = clock64();
         long long prof[4] = {0, 0, 0, 0};
+        long long ph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
             const int h = (int)(w / n_items);
             const WorkItem it = items[w % n_items];
-            const bool active = qt * BM < it.nrows;  // an inactive query tile only keeps the barriers in step
+            const bool active = qt * BM < it.nrows && !((dbg & 16) && qt == 1);  // an inactive query tile only keeps the barriers in step
             const int local = qt * BM + quarter * 32 + lane;
             const bool rvalid = local < it.nrows;
             if (active) row_init<KG>(rs, wl, k, lane, rvalid);
@@ -421,33 +425,50 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     float sub[16], quad[4];
                     uint32_t v[64];
                     const bool ragged = ncol < BN;
+                    long long s0 = 0, s1 = 0, s2 = 0, s3 = 0, s4 = 0;
+                    if (dbg & 32) s0 = clock64();
                     if (active) {
                         ptx::tmem_ld_32x64_sync(taddr, v);
+                        if (dbg & 32) s1 = clock64();
                         if (!(dbg & 2)) {
                             if (ragged) half_maxima<true>(v, ncol, sub, quad);
                             else half_maxima<false>(v, ncol, sub, quad);
                         }
+                        if (dbg & 32) s2 = clock64();
                         ptx::tmem_ld_32x64_sync(taddr + 64, v);
+                        if (dbg & 32) s3 = clock64();
                     }
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
+                    if (dbg & 32) { s4 = clock64(); ph[0] += s0 - c1; ph[1] += s1 - s0; ph[2] += s2 - s1; ph[3] += s3 - s2; ph[4] += s4 - s3; }
                     if (active && !(dbg & 2)) {
                         if (ragged) half_maxima<true>(v, ncol - 64, sub + 8, quad + 2);
                         else half_maxima<false>(v, ncol - 64, sub + 8, quad + 2);
                         const float gm = fmaxf(fmaxf(quad[0], quad[1]), fmaxf(quad[2], quad[3]));
+                        if (dbg & 32) { if (gm == 77.125f) rs.tau = 1.0f; ph[5] += clock64() - s4; }
                         if (!(dbg & 1)) {
                             const long long p0 = (dbg & 8) ? clock64() : 0;
+                            // A flush by one warp stalls the other seven within two tiles (the accumulator
+                            // buffers are only two deep), so the warps flush together: whoever must flush
+                            // bumps a CTA-wide counter and every warp that sees it move flushes at its next tile.
+                            const int req = *sFlushReq;
+                            bool do_flush = req != flush_seen;
                             if (__any_sync(FULL, gm > rs.tau)) {  // some lane of the warp has a hit in this tile
                                 uint32_t pend = wp_addr + (uint32_t)rs.cnt * 256u;
                                 append_groups(sub, quad, rs.tau, key0, pend);
                                 rs.cnt = (int)((pend - wp_addr) >> 8);
                                 if (dbg & 8) { prof[0] += clock64() - p0; ++prof[1]; }
                                 if (__any_sync(FULL, rs.cnt > ROOM - 16)) {  // a tile adds at most 16 groups per row
-                                    const long long p1 = (dbg & 8) ? clock64() : 0;
-                                    flush_pending<KG>(rs, wl, wp, lane, rvalid);
-                                    if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
+                                    do_flush = true;
+                                    if (lane == 0 && req == flush_seen) atomicAdd(const_cast<int*>(sFlushReq), 1);
                                 }
+                            }
+                            if (do_flush) {
+                                const long long p1 = (dbg & 8) ? clock64() : 0;
+                                flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                                flush_seen = req + ((req == flush_seen) ? 1 : 0);
+                                if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
                             }
                         } else if (gm == 123.456f) {
                             rs.tau = 0.0f;  // timing experiment: keep the maxima alive
@@ -482,6 +503,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             timing[blockIdx.x * 8 + 6] = t_work;
             timing[blockIdx.x * 8 + 7] = tcnt;
             for (int i = 0; i < 4; ++i) timing[148 * 8 + blockIdx.x * 8 + i] = prof[i];
+            for (int i = 0; i < 8; ++i) timing[148 * 16 + blockIdx.x * 8 + i] = ph[i];
         }
     }
 
