@@ -86,7 +86,7 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     if (ev) cudaEventRecord(ev[1], a.stream);
     if ((tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], a.stream);
-    if (tc && launch_refine_topk(a) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (tc && launch_refine_topk(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[3], a.stream);
     if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4], a.stream);

@@ -227,6 +227,42 @@ __device__ __forceinline__ void accumulate_hit(int e, int HK, int h, int H, int 
     }
 }
 
+// Accumulates the hits first, first+stride, ... (< len) of one list; four hits are in flight at a time
+// so that the dependent loads (pair id -> weights and rows) of different hits overlap.
+template <typename T, int D>
+__device__ __forceinline__ void accumulate_list(const int* __restrict__ list, int first, int stride, int len, int HK,
+                                                int h, int H, int part, const T* __restrict__ Q,
+                                                const T* __restrict__ dOut, const float* __restrict__ ws_p,
+                                                const float* __restrict__ ws_ds, float (&accV)[Elem<T>::kVec],
+                                                float (&accK)[Elem<T>::kVec]) {
+    constexpr int VEC = Elem<T>::kVec;
+    int t = first;
+    for (; t + 3 * stride < len; t += 4 * stride) {
+        int e[4];
+        float pw[4], dsw[4], gv[4][VEC], qv[4][VEC];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) e[u] = __ldg(list + t + u * stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const size_t off = ((size_t)(e[u] / HK) * H + h) * D + part * VEC;
+            pw[u] = __ldg(ws_p + e[u]);
+            dsw[u] = __ldg(ws_ds + e[u]);
+            Elem<T>::load_vec(dOut + off, gv[u]);
+            Elem<T>::load_vec(Q + off, qv[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int c = 0; c < VEC; ++c) {
+                accV[c] = fmaf(pw[u], gv[u][c], accV[c]);
+                accK[c] = fmaf(dsw[u], qv[u][c], accK[c]);
+            }
+        }
+    }
+    for (; t < len; t += stride)
+        accumulate_hit<T, D>(__ldg(list + t), HK, h, H, part, Q, dOut, ws_p, ws_ds, accV, accK);
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 bwd_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
@@ -246,8 +282,7 @@ bwd_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
         float accV[VEC], accK[VEC];
 #pragma unroll
         for (int c = 0; c < VEC; ++c) { accV[c] = 0.0f; accK[c] = 0.0f; }
-        for (int t = sub; t < len; t += EPW)
-            accumulate_hit<T, D>(__ldg(pairs + start + t), HK, h, H, part, Q, dOut, ws_p, ws_ds, accV, accK);
+        accumulate_list<T, D>(pairs + start, sub, EPW, len, HK, h, H, part, Q, dOut, ws_p, ws_ds, accV, accK);
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
@@ -284,8 +319,8 @@ bwd_long_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
         float accV[VEC], accK[VEC];
 #pragma unroll
         for (int c = 0; c < VEC; ++c) { accV[c] = 0.0f; accK[c] = 0.0f; }
-        for (int t = wid * EPW + sub; t < len; t += kWarpsPerBlock * EPW)
-            accumulate_hit<T, D>(__ldg(pairs + start + t), HK, h, H, part, Q, dOut, ws_p, ws_ds, accV, accK);
+        accumulate_list<T, D>(pairs + start, wid * EPW + sub, kWarpsPerBlock * EPW, len, HK, h, H, part, Q, dOut, ws_p,
+                              ws_ds, accV, accK);
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
@@ -355,7 +390,7 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
 
     bwd_segments_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         Q, dOut, ws_p, ws_ds, seg_off, pairs, n_rows, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
-    bwd_long_segments_kernel<T, D><<<148 * 4, kWarpsPerBlock * 32, 0, a.stream>>>(
+    bwd_long_segments_kernel<T, D><<<148 * 8, kWarpsPerBlock * 32, 0, a.stream>>>(
         Q, dOut, ws_p, ws_ds, seg_off, pairs, long_list, sb, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
     if (ev) cudaEventRecord(ev[2], a.stream);
     return cudaGetLastError();

@@ -174,7 +174,7 @@ void set_score_select_fault_test(int drop_first_tile, long long wait_limit_cycle
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump);
 // refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k
-cudaError_t launch_refine_topk(const FwdArgs& a);
+cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w);
 // epilogue.cu: softmax over the k kept scores fused with the gather-V weighted sum
 cudaError_t launch_softmax_gather(const FwdArgs& a);
 // backward.cu

@@ -30,12 +30,12 @@ __device__ inline int graph_end(const int32_t* offs, int G, int N, int i) {
 
 template <typename T, int D, int E>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ K, const int32_t* __restrict__ offs, int G,
+refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int32_t* __restrict__ offs, int G,
                    int N, int H, int k, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
                    const StatusBlock* __restrict__ sb) {
     if (sb->status != KMIP_OK) return;
     constexpr int CAP = 32 * E;
-    constexpr int VEC = Elem<T>::kVec;
+    static_assert(sizeof(T) == 2, "the rescoring kernel reads bf16 keys");
     __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
     __shared__ float s_q[kWarpsPerBlock][D];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -75,33 +75,52 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ K, const int32
 
         float tau = floor_tau;
         int cnt = 0;
-        for (int t0 = 0; t0 < k; t0 += 32 / kGroup) {
-            const int t = t0 + lane / kGroup;
-            int g = -1;
+        constexpr int GPR = 32 / kGroup;           // groups scored per step (one key per lane)
+        constexpr int NV = D * (int)sizeof(T) / 16;  // 16-byte vectors per key row
+        constexpr int U = (NV <= 8) ? 2 : 1;       // steps whose loads are issued together
+        for (int t0 = 0; t0 < k; t0 += U * GPR) {
+            int jj[U];
+            bool valid[U];
+            uint4 raw[U][NV];
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (e == (t0 >> 5)) g = __shfl_sync(0xFFFFFFFFu, gid[e], t & 31);
-            const int j = g + (lane % kGroup);
-            const bool valid = t < k && g >= 0 && j < hi;
-            float s = 0.0f;
-            if (valid) {
-                const T* kr = K + ((size_t)j * H + h) * D;
+            for (int u = 0; u < U; ++u) {
+                const int tb = t0 + u * GPR, t = tb + lane / kGroup;
+                int g = -1;
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += VEC) {
-                    float kv[VEC];
-                    Elem<T>::load_vec(kr + c0, kv);
+                for (int e = 0; e < 4; ++e)
+                    if (e == (tb >> 5)) g = __shfl_sync(0xFFFFFFFFu, gid[e], t & 31);
+                jj[u] = g + (lane % kGroup);
+                valid[u] = t < k && g >= 0 && jj[u] < hi;
+                if (valid[u]) {
+                    // keys regrouped by head: the 8 keys of a group are 8 consecutive rows
+                    const uint4* kr = reinterpret_cast<const uint4*>(Kp + ((size_t)h * N + jj[u]) * D);
 #pragma unroll
-                    for (int c = 0; c < VEC; ++c) s = fmaf(q[c0 + c], kv[c], s);
+                    for (int v = 0; v < NV; ++v) raw[u][v] = __ldg(kr + v);
                 }
             }
-            const bool pass = valid && (s > tau);
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, pass);
-            if (m) {
-                if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, j);
-                cnt += __popc(m);
-                if (cnt > room - 32) {
-                    tau = fmaxf(floor_tau, warp_compact_row<E>(row, k, cnt, lane));
-                    cnt = 0;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float s = 0.0f;
+                if (valid[u]) {
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        const uint32_t wv[4] = {raw[u][v].x, raw[u][v].y, raw[u][v].z, raw[u][v].w};
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            s = fmaf(q[v * 8 + 2 * x], __uint_as_float(wv[x] << 16), s);
+                            s = fmaf(q[v * 8 + 2 * x + 1], __uint_as_float(wv[x] & 0xFFFF0000u), s);
+                        }
+                    }
+                }
+                const bool pass = valid[u] && (s > tau);
+                const unsigned m = __ballot_sync(0xFFFFFFFFu, pass);
+                if (m) {
+                    if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, jj[u]);
+                    cnt += __popc(m);
+                    if (cnt > room - 32) {
+                        tau = fmaxf(floor_tau, warp_compact_row<E>(row, k, cnt, lane));
+                        cnt = 0;
+                    }
                 }
             }
         }
@@ -111,13 +130,13 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ K, const int32
 }
 
 template <int D>
-cudaError_t launch_d(const FwdArgs& a) {
+cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w) {
     using T = __nv_bfloat16;
     const long long n_rows = (long long)a.N * a.H;
     const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
 #define KMIP_LAUNCH_REFINE(E_) \
     refine_topk_kernel<T, D, E_><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
-        static_cast<const T*>(a.Q), static_cast<const T*>(a.K), a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
+        static_cast<const T*>(a.Q), reinterpret_cast<const T*>(a.ws + w.kpack_off), a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
         a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws))
     // pending room CAP-k >= 96, so that the survivors of a row (rarely more than 2k) fit without
     // intermediate compactions
@@ -129,12 +148,12 @@ cudaError_t launch_d(const FwdArgs& a) {
 
 }  // namespace
 
-cudaError_t launch_refine_topk(const FwdArgs& a) {
+cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w) {
     switch (a.d) {
-        case 16: return launch_d<16>(a);
-        case 32: return launch_d<32>(a);
-        case 64: return launch_d<64>(a);
-        case 128: return launch_d<128>(a);
+        case 16: return launch_d<16>(a, w);
+        case 32: return launch_d<32>(a, w);
+        case 64: return launch_d<64>(a, w);
+        case 128: return launch_d<128>(a, w);
         default: return cudaErrorInvalidValue;
     }
 }
