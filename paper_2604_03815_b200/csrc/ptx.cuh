@@ -68,12 +68,15 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t par
 // when `abort_flag` (shared memory) is set by another thread or after roughly `limit_cycles` SM
 // clocks (about 4 s by default), in which case it sets the flag itself and returns false.
 // Callers leave their loops on false; nothing waits forever.
+// SLEEP_NS > 0 adds a sleep between polls, for waiters that can afford a late wake-up.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   long long limit_cycles = 8000000000ll) {
     if (mbar_try_wait(bar, parity)) return true;
     uint32_t spins = 0;
     long long t0 = 0;
     while (!mbar_try_wait_suspend(bar, parity, 20000u)) {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
         if ((++spins & 15u) == 0u) {
             if (*abort_flag) return false;
             const long long now = clock64();

@@ -81,13 +81,15 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                 ((uint32_t)(BM >> 4) << 24);
 
-constexpr int ROOM = 32;  // pending candidate slots per row
+constexpr int kRelaxedPollNs = 100;  // sleep between polls of the waits that are off the critical path
+constexpr int NBUF = 4;  // accumulator buffers of BN columns: all 512 columns of tensor memory, used as a ring
 
 template <int KG, int NQT, int S>
 struct SmemPlan {
-    static constexpr int LIST = 8 * KG;          // list slots per row (k <= LIST)
-    static constexpr int SLOTS = LIST + ROOM;    // cand_t per row
-    static constexpr int NBARS = 3 + 2 * S + 4;
+    static constexpr int LIST = 8 * KG;               // list slots per row (k <= LIST)
+    static constexpr int ROOM = NQT >= 3 ? 24 : 32;   // pending candidate slots per row (a tile adds at most 16)
+    static constexpr int SLOTS = LIST + ROOM;         // cand_t per row
+    static constexpr int NBARS = 3 + 2 * S + 2 * NBUF;
 };
 
 struct Bars {
@@ -99,12 +101,15 @@ struct Bars {
     __device__ uint32_t k_full(int s) const { return base + 8 * (3 + s); }
     __device__ uint32_t k_empty(int s) const { return base + 8 * (3 + S + s); }
     __device__ uint32_t t_full(int b) const { return base + 8 * (3 + 2 * S + b); }
-    __device__ uint32_t t_empty(int b) const { return base + 8 * (3 + 2 * S + 2 + b); }
+    __device__ uint32_t t_empty(int b) const { return base + 8 * (3 + 2 * S + NBUF + b); }
 };
 
+// SLEEP_NS > 0: the waiter is off the critical path (the TMA producer and the MMA issuers run
+// well ahead of the selection warps) and sleeps between polls instead of competing for issue slots.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                               StatusBlock* sb, int who, long long limit) {
-    if (ptx::mbar_wait_bounded(bar, parity, abort_flag, limit)) return true;
+    if (ptx::mbar_wait_bounded<SLEEP_NS>(bar, parity, abort_flag, limit)) return true;
     record_status(sb, KMIP_ERR_TIMEOUT, who);
     return false;
 }
@@ -223,7 +228,7 @@ __device__ __forceinline__ void append_groups(const float (&sub)[16], const floa
 }
 
 template <int D, int KG, int NQT, int S, bool DUMP>
-__global__ void __launch_bounds__(NQT * 128 + 96, 1)
+__global__ void __launch_bounds__(NQT * 128 + 32 + 32 * (NQT >= 3 ? 1 : 2), 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
@@ -233,7 +238,9 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
     constexpr int NEPI = 4 * NQT;
-    constexpr uint32_t TMEM_COLS = NQT * 2 * BN;
+    constexpr int NISS = NQT >= 3 ? 1 : 2;  // MMA issuer threads (see the issuer branch)
+    constexpr int ROOM = Sp::ROOM;
+    constexpr uint32_t TMEM_COLS = NBUF * BN;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -250,15 +257,15 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bars.q_full(), 1);
-        ptx::mbar_init(bars.q_empty(), 2);  // both MMA issuers commit to it
-        ptx::mbar_init(bars.done(), 2);
+        ptx::mbar_init(bars.q_empty(), NISS);  // every MMA issuer commits to it
+        ptx::mbar_init(bars.done(), NISS);
         for (int s = 0; s < S; ++s) {
             ptx::mbar_init(bars.k_full(s), 1);
-            ptx::mbar_init(bars.k_empty(s), 1);
+            ptx::mbar_init(bars.k_empty(s), NQT);  // one arrival per query tile
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < NBUF; ++b) {
             ptx::mbar_init(bars.t_full(b), 1);
-            ptx::mbar_init(bars.t_empty(b), NEPI);  // one arrival per selection warp
+            ptx::mbar_init(bars.t_empty(b), 4);  // the four selection warps of the buffer's query tile
         }
         *sAbort = 0;
         *sFlushReq = 0;
@@ -289,7 +296,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const int h = (int)(w / n_items);
                 const WorkItem it = items[w % n_items];
-                if (!(ok = wait_or_abort(bars.q_empty(), (ic & 1) ^ 1, sAbort, sb, 1, wait_limit))) break;
+                if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.q_empty(), (ic & 1) ^ 1, sAbort, sb, 1, wait_limit))) break;
                 ptx::mbar_arrive_expect_tx(bars.q_full(), NQT * Sh::TILE_BYTES);
                 for (int qt = 0; qt < NQT; ++qt)
                     for (int ch = 0; ch < Sh::KCH; ++ch)
@@ -298,7 +305,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
                 for (int j = 0; j < ntiles; ++j, ++kt) {
                     const int s = kt % S;
-                    if (!(ok = wait_or_abort(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit))) break;
+                    if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit))) break;
                     // failure-detection test hook: CTA 0 never loads its first key tile, so the waits on
                     // that stage must run out, be reported and leave the context usable
                     if (drop_first_tile && blockIdx.x == 0 && kt == 0) continue;
@@ -319,44 +326,63 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 }
             }
         }
-    } else if (warp == NEPI + 1 || warp == NEPI + 2) {
+    } else if (warp >= NEPI + 1 && warp <= NEPI + NISS) {
         // ------------------------------------------------------------------ MMA issuers
-        // Two threads in two warps: issuer p takes the key tiles with running number kt = p (mod 2),
-        // i.e. accumulator buffer p, so the barrier waits and the commit of one overlap with the
-        // MMAs of the other.  Per tile an issuer runs the MMAs of every query tile and commits
-        // once; the commit tells the selection warps that the scores are ready and (forwarded by
-        // selection warp 0) that the key stage can be refilled.
+        // The (key tile, query tile) pairs of the CTA form one sequence; pair number q uses
+        // accumulator buffer q mod 4, so the issue side runs up to four pairs ahead of the slowest
+        // selection warp group, and the commit after a pair's MMAs tells that pair's selection
+        // warps that the scores are ready.  With one or two query tiles two threads in two warps
+        // take the pairs alternately (the barrier waits and the commit of one overlap with the
+        // MMAs of the other); every buffer is then filled by one issuer and read by one warp
+        // group.  With three query tiles a warp group meets a buffer only every third time it is
+        // filled, and a parity wait is only sound if the fill before the awaited one has completed;
+        // a single issuer completes the pairs in order, which guarantees that.
         if (lane == 0) {
             const int mine = warp - (NEPI + 1);
+            // operand descriptors: the query tiles stay put, the key stages differ only in the start address
+            uint64_t desc_q[NQT][Sh::KSTEPS], desc_k0[Sh::KSTEPS];
+#pragma unroll
+            for (int ks = 0; ks < Sh::KSTEPS; ++ks) {
+                const int off = (ks / Sh::STEPS_PER_CH) * Sh::CH_BYTES + (ks % Sh::STEPS_PER_CH) * 32;
+#pragma unroll
+                for (int qt = 0; qt < NQT; ++qt) desc_q[qt][ks] = make_smem_desc<D>(ptx::smem_u32(sQ + qt * Sh::TILE_BYTES + off));
+                desc_k0[ks] = make_smem_desc<D>(ptx::smem_u32(sK + off));
+            }
             int kt = 0, ic = 0;
             bool ok = true;
             long long w_kfull = 0, w_tempty = 0, t_begin = clock64();
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem it = items[w % n_items];
-                const int nq = (NQT == 2 && it.nrows > BM && !(dbg & 16)) ? 2 : 1;  // dbg 16: timing experiment, one query tile only
-                if (!(ok = wait_or_abort(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
+                const int nq = (it.nrows + BM - 1) / BM;  // query tiles of the item that hold rows
+                if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
                 ptx::tc_fence_after();
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
-                for (int j = 0; j < ntiles; ++j, ++kt) {
-                    const int s = kt % S, b = kt & 1;
-                    if (b != mine) continue;
-                    long long c0 = (dbg & 8) ? clock64() : 0;
-                    if (!(ok = wait_or_abort(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
-                    long long c1 = (dbg & 8) ? clock64() : 0;
-                    if (!(ok = wait_or_abort(bars.t_empty(b), ((kt >> 1) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
-                    if (dbg & 8) { w_kfull += c1 - c0; w_tempty += clock64() - c1; }
-                    ptx::tc_fence_after();
-                    for (int qt = 0; qt < nq; ++qt) {
-                        const uint32_t d_tmem = tmem_base + (uint32_t)((qt * 2 + b) * BN);
+                for (int j = 0; ok && j < ntiles; ++j, ++kt) {
+                    const int s = kt % S;
+                    const uint64_t stage_off = (uint64_t)((s * Sh::TILE_BYTES) >> 4);  // start-address field counts 16-byte units
+                    bool have_keys = false;
 #pragma unroll
-                        for (int ks = 0; ks < Sh::KSTEPS; ++ks) {
-                            const int off = (ks / Sh::STEPS_PER_CH) * Sh::CH_BYTES + (ks % Sh::STEPS_PER_CH) * 32;
-                            const uint64_t da = make_smem_desc<D>(ptx::smem_u32(sQ + qt * Sh::TILE_BYTES + off));
-                            const uint64_t db = make_smem_desc<D>(ptx::smem_u32(sK + s * Sh::TILE_BYTES + off));
-                            ptx::mma_bf16_ss(d_tmem, da, db, kInstrDesc, ks > 0 ? 1u : 0u);
+                    for (int qt = 0; qt < NQT; ++qt) {
+                        const int seq = kt * NQT + qt;
+                        if (NISS == 2 && (seq & 1) != mine) continue;
+                        const int b = seq & (NBUF - 1);
+                        long long c0 = (dbg & 8) ? clock64() : 0;
+                        if (!have_keys) {
+                            if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
+                            have_keys = true;
                         }
+                        long long c1 = (dbg & 8) ? clock64() : 0;
+                        if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.t_empty(b), ((seq >> 2) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
+                        if (dbg & 8) { w_kfull += c1 - c0; w_tempty += clock64() - c1; }
+                        ptx::tc_fence_after();
+                        if (qt < nq) {
+                            const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
+#pragma unroll
+                            for (int ks = 0; ks < Sh::KSTEPS; ++ks)
+                                ptx::mma_bf16_ss(d_tmem, desc_q[qt][ks], desc_k0[ks] + stage_off, kInstrDesc, ks > 0 ? 1u : 0u);
+                        }
+                        ptx::mma_commit(bars.t_full(b));
                     }
-                    ptx::mma_commit(bars.t_full(b));
                 }
                 if (!ok) break;
                 ptx::mma_commit(bars.q_empty());
@@ -389,36 +415,41 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
             const int h = (int)(w / n_items);
             const WorkItem it = items[w % n_items];
-            const bool active = qt * BM < it.nrows && !((dbg & 16) && qt == 1);  // an inactive query tile only keeps the barriers in step
+            const bool active = qt * BM < it.nrows;  // an inactive query tile only keeps the barriers in step
             const int local = qt * BM + quarter * 32 + lane;
             const bool rvalid = local < it.nrows;
             if (active) row_init<KG>(rs, wl, k, lane, rvalid);
             __syncwarp();
             const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
             for (int j = 0; j < ntiles; ++j, ++tcnt) {
-                const int b = tcnt & 1;
+                const int seq = tcnt * NQT + qt;  // this warp group's (key tile, query tile) pair
+                const int b = seq & (NBUF - 1);
                 const long long c0 = (dbg & 8) ? clock64() : 0;
-                ok = wait_or_abort(bars.t_full(b), (tcnt >> 1) & 1, sAbort, sb, 6, wait_limit);
+                ok = wait_or_abort(bars.t_full(b), (seq >> 2) & 1, sAbort, sb, 6, wait_limit);
                 ok = __all_sync(FULL, ok);
                 if (!ok) break;
                 const long long c1 = (dbg & 8) ? clock64() : 0;
-                // the tile's MMAs have retired, so its key stage can be refilled
-                if (warp == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
+                // this query tile's MMAs on the key tile have retired; once that holds for every query
+                // tile the key stage can be refilled
+                if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
                 ptx::tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((qt * 2 + b) * BN);
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * BN);
                 const int key0 = it.key_lo + j * BN;
                 const int ncol = min(BN, it.key_hi - key0);
                 if (DUMP) {
-                    uint32_t v[BN];
-                    if (active) ptx::tmem_ld_32x128_sync(taddr, v);
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        uint32_t v[32];
+                        ptx::tmem_ld_32x32_sync(taddr + c * 32, v);
+                        if (active && rvalid)
+#pragma unroll
+                            for (int x = 0; x < 32; ++x)
+                                if (c * 32 + x < ncol)
+                                    dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + c * 32 + x] = __uint_as_float(v[x]);
+                    }
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
-                    if (active && rvalid)
-#pragma unroll
-                        for (int x = 0; x < BN; ++x)
-                            if (x < ncol)
-                                dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + x] = __uint_as_float(v[x]);
                 } else {
                     // two 64-column halves keep the register footprint small; the accumulator buffer
                     // goes back to the MMA issuer as soon as the second half is in registers
@@ -584,7 +615,7 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     if (err != cudaSuccess) return err;
     const long long max_total = (long long)w.max_items * a.H;
     const int grid = (int)std::min<long long>(sm_count(), max_total);
-    kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
+    kern<<<grid, NQT * 128 + 32 + 32 * (NQT >= 3 ? 1 : 2), smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
         a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing, g_wait_limit_cycles,
         g_drop_first_tile);
@@ -595,7 +626,7 @@ template <int D, bool DUMP>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     // (list groups KG, query tiles per CTA, key stages) by k and head width; shared memory decides
     if (a.k <= 32) {
-        if constexpr (D <= 32) return launch_cfg<D, 4, 2, 6, DUMP>(a, w, dump);
+        if constexpr (D <= 32) return launch_cfg<D, 4, 3, 4, DUMP>(a, w, dump);
         else if constexpr (D == 64) return launch_cfg<D, 4, 2, 3, DUMP>(a, w, dump);
         else return launch_cfg<D, 4, 1, 3, DUMP>(a, w, dump);
     }
@@ -638,7 +669,7 @@ bool score_select_tc_supported(int32_t d, int32_t k) {
     return k <= 128 && d <= 64;
 }
 
-int score_select_tc_rows_per_item(int32_t d, int32_t k) { return (k <= 32 && d <= 64) ? 256 : 128; }  // 128 * query tiles per CTA
+int score_select_tc_rows_per_item(int32_t d, int32_t k) { return k > 32 || d > 64 ? 128 : d > 32 ? 256 : 384; }  // 128 * query tiles per CTA
 
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w) {
     return launch_any<false>(a, w, nullptr);
