@@ -89,19 +89,20 @@ struct SmemPlan {
     static constexpr int LIST = 8 * KG;               // list slots per row (k <= LIST)
     static constexpr int ROOM = NQT >= 3 ? 24 : 32;   // pending candidate slots per row (a tile adds at most 16)
     static constexpr int SLOTS = LIST + ROOM;         // cand_t per row
-    static constexpr int NBARS = 3 + 2 * S + 2 * NBUF;
+    static constexpr int PERIOD = NQT == 3 ? 12 : 4;  // pairs between two uses of a buffer by the same query tile
+    static constexpr int NBARS = 3 + 2 * S + NBUF * NQT + NBUF;
 };
 
 struct Bars {
     uint32_t base;
-    int S;
+    int S, NQT;
     __device__ uint32_t q_full() const { return base; }
     __device__ uint32_t q_empty() const { return base + 8; }
     __device__ uint32_t done() const { return base + 16; }
     __device__ uint32_t k_full(int s) const { return base + 8 * (3 + s); }
     __device__ uint32_t k_empty(int s) const { return base + 8 * (3 + S + s); }
-    __device__ uint32_t t_full(int b) const { return base + 8 * (3 + 2 * S + b); }
-    __device__ uint32_t t_empty(int b) const { return base + 8 * (3 + 2 * S + NBUF + b); }
+    __device__ uint32_t t_full(int b, int qt) const { return base + 8 * (3 + 2 * S + b * NQT + qt); }
+    __device__ uint32_t t_empty(int b) const { return base + 8 * (3 + 2 * S + NBUF * NQT + b); }
 };
 
 // SLEEP_NS > 0: the waiter is off the critical path (the TMA producer and the MMA issuers run
@@ -228,7 +229,7 @@ __device__ __forceinline__ void append_groups(const float (&sub)[16], const floa
 }
 
 template <int D, int KG, int NQT, int S, bool DUMP>
-__global__ void __launch_bounds__(NQT * 128 + 32 + 32 * (NQT >= 3 ? 1 : 2), 1)
+__global__ void __launch_bounds__(NQT * 128 + 96, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
@@ -238,7 +239,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
     constexpr int NEPI = 4 * NQT;
-    constexpr int NISS = NQT >= 3 ? 1 : 2;  // MMA issuer threads (see the issuer branch)
+    constexpr int NISS = 2;  // MMA issuer threads (see the issuer branch)
     constexpr int ROOM = Sp::ROOM;
     constexpr uint32_t TMEM_COLS = NBUF * BN;
 
@@ -253,7 +254,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     volatile int* sFlushReq = reinterpret_cast<volatile int*>(sTmem + 2);  // CTA-wide flush request counter
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    Bars bars{ptx::smem_u32(sBars), S};
+    Bars bars{ptx::smem_u32(sBars), S, NQT};
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bars.q_full(), 1);
@@ -264,8 +265,8 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ptx::mbar_init(bars.k_empty(s), NQT);  // one arrival per query tile
         }
         for (int b = 0; b < NBUF; ++b) {
-            ptx::mbar_init(bars.t_full(b), 1);
-            ptx::mbar_init(bars.t_empty(b), 4);  // the four selection warps of the buffer's query tile
+            for (int q = 0; q < NQT; ++q) ptx::mbar_init(bars.t_full(b, q), 1);
+            ptx::mbar_init(bars.t_empty(b), 4);  // the four selection warps of the query tile that read the buffer
         }
         *sAbort = 0;
         *sFlushReq = 0;
@@ -330,13 +331,12 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // ------------------------------------------------------------------ MMA issuers
         // The (key tile, query tile) pairs of the CTA form one sequence; pair number q uses
         // accumulator buffer q mod 4, so the issue side runs up to four pairs ahead of the slowest
-        // selection warp group, and the commit after a pair's MMAs tells that pair's selection
-        // warps that the scores are ready.  With one or two query tiles two threads in two warps
-        // take the pairs alternately (the barrier waits and the commit of one overlap with the
-        // MMAs of the other); every buffer is then filled by one issuer and read by one warp
-        // group.  With three query tiles a warp group meets a buffer only every third time it is
-        // filled, and a parity wait is only sound if the fill before the awaited one has completed;
-        // a single issuer completes the pairs in order, which guarantees that.
+        // selection warp group.  Two threads in two warps take the pairs alternately, so the
+        // barrier waits and the commit of one overlap with the MMAs of the other; a buffer is always
+        // filled by the same issuer.  The commit after a pair's MMAs tells that pair's selection
+        // warps that the scores are ready.  It goes to a barrier of its own per (buffer, query
+        // tile): with three query tiles a warp group meets a buffer only every third time it is
+        // filled, and a parity wait is sound only on a barrier whose every phase the waiter sees.
         if (lane == 0) {
             const int mine = warp - (NEPI + 1);
             // operand descriptors: the query tiles stay put, the key stages differ only in the start address
@@ -364,7 +364,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
                     for (int qt = 0; qt < NQT; ++qt) {
                         const int seq = kt * NQT + qt;
-                        if (NISS == 2 && (seq & 1) != mine) continue;
+                        if ((seq & 1) != mine) continue;
                         const int b = seq & (NBUF - 1);
                         long long c0 = (dbg & 8) ? clock64() : 0;
                         if (!have_keys) {
@@ -381,7 +381,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                             for (int ks = 0; ks < Sh::KSTEPS; ++ks)
                                 ptx::mma_bf16_ss(d_tmem, desc_q[qt][ks], desc_k0[ks] + stage_off, kInstrDesc, ks > 0 ? 1u : 0u);
                         }
-                        ptx::mma_commit(bars.t_full(b));
+                        ptx::mma_commit(bars.t_full(b, qt));
                     }
                 }
                 if (!ok) break;
@@ -425,7 +425,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 const int seq = tcnt * NQT + qt;  // this warp group's (key tile, query tile) pair
                 const int b = seq & (NBUF - 1);
                 const long long c0 = (dbg & 8) ? clock64() : 0;
-                ok = wait_or_abort(bars.t_full(b), (seq >> 2) & 1, sAbort, sb, 6, wait_limit);
+                ok = wait_or_abort(bars.t_full(b, qt), (seq / Sp::PERIOD) & 1, sAbort, sb, 6, wait_limit);
                 ok = __all_sync(FULL, ok);
                 if (!ok) break;
                 const long long c1 = (dbg & 8) ? clock64() : 0;
@@ -615,7 +615,7 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     if (err != cudaSuccess) return err;
     const long long max_total = (long long)w.max_items * a.H;
     const int grid = (int)std::min<long long>(sm_count(), max_total);
-    kern<<<grid, NQT * 128 + 32 + 32 * (NQT >= 3 ? 1 : 2), smem_bytes, a.stream>>>(
+    kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
         a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing, g_wait_limit_cycles,
         g_drop_first_tile);
