@@ -208,9 +208,13 @@ __device__ __forceinline__ void half_maxima(uint32_t (&v)[64], int nvalid, float
 // lane's next free slot (256 bytes apart).
 __device__ __forceinline__ void append_groups(const float (&sub)[16], const float (&quad)[4], float tau, int key_base,
                                               uint32_t& pend) {
+    // four independent votes first, warp-uniform branches afterwards
+    unsigned hit[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) hit[c] = __ballot_sync(FULL, quad[c] > tau);
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        if (__any_sync(FULL, quad[c] > tau)) {
+        if (hit[c]) {
 #pragma unroll
             for (int g = 4 * c; g < 4 * c + 4; ++g) {
                 asm volatile(
