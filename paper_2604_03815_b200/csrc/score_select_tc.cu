@@ -358,7 +358,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem it = items[w % n_items];
                 const int nq = (it.nrows + BM - 1) / BM;  // query tiles of the item that hold rows
-                if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
+                if (!(ok = wait_or_abort<0>(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
                 ptx::tc_fence_after();
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
                 for (int j = 0; ok && j < ntiles; ++j, ++kt) {
@@ -372,11 +372,11 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         const int b = seq & (NBUF - 1);
                         long long c0 = (dbg & 8) ? clock64() : 0;
                         if (!have_keys) {
-                            if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
+                            if (!(ok = wait_or_abort<0>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
                             have_keys = true;
                         }
                         long long c1 = (dbg & 8) ? clock64() : 0;
-                        if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.t_empty(b), ((seq >> 2) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
+                        if (!(ok = wait_or_abort<0>(bars.t_empty(b), ((seq >> 2) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
                         if (dbg & 8) { w_kfull += c1 - c0; w_tempty += clock64() - c1; }
                         ptx::tc_fence_after();
                         if (qt < nq) {
@@ -429,9 +429,14 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 const int seq = tcnt * NQT + qt;  // this warp group's (key tile, query tile) pair
                 const int b = seq & (NBUF - 1);
                 const long long c0 = (dbg & 8) ? clock64() : 0;
-                ok = wait_or_abort(bars.t_full(b, qt), (seq / Sp::PERIOD) & 1, sAbort, sb, 6, wait_limit);
-                ok = __all_sync(FULL, ok);
-                if (!ok) break;
+                if (!__all_sync(FULL, ptx::mbar_try_wait(bars.t_full(b, qt), (seq / Sp::PERIOD) & 1))) {
+                    // The scores are not ready yet: use the wait to merge pending candidates into the
+                    // lists (always allowed, and it raises the thresholds early), then block.
+                    if (!DUMP && active && !(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                    ok = wait_or_abort(bars.t_full(b, qt), (seq / Sp::PERIOD) & 1, sAbort, sb, 6, wait_limit);
+                    ok = __all_sync(FULL, ok);
+                    if (!ok) break;
+                }
                 const long long c1 = (dbg & 8) ? clock64() : 0;
                 // this query tile's MMAs on the key tile have retired; once that holds for every query
                 // tile the key stage can be refilled
