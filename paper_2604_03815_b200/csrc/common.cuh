@@ -25,11 +25,11 @@ struct StatusBlock {
 };
 static_assert(sizeof(StatusBlock) == kStatusBytes, "status block size");
 
-// One unit of work of the tensor-core score kernel: up to 256 consecutive query rows of one
+// One unit of work of the tensor-core score kernel: up to 384 consecutive query rows of one
 // graph and that graph's key range (Eq. 1 restricted to the graph by the CSR offsets).
 struct WorkItem {
     int row0;    // first query row
-    int nrows;   // 1..256
+    int nrows;   // 1..384 (128 x the query tiles per CTA of the launched configuration)
     int key_lo;  // graph's first row
     int key_hi;  // one past the graph's last row
 };

@@ -209,17 +209,19 @@ def make_config(i: int, **kw) -> Workload:
 
 
 def sample_rows(w: Workload, n: int, seed: int = 12345) -> np.ndarray:
-    """A stratified, seeded sample of query rows: first/last rows of each graph and of
-    256-row blocks, plus uniform picks; sorted, unique, int64."""
+    """A stratified, seeded sample of query rows: first/last rows of each graph and of its
+    128-, 256- and 384-row blocks, plus uniform picks; sorted, unique, int64."""
     offs = w.graph_offsets.astype(np.int64)
     picks = []
     for g in range(w.G):
         lo, hi = offs[g], offs[g + 1]
         if hi > lo:
             picks += [lo, hi - 1, min(lo + 127, hi - 1), min(lo + 128, hi - 1),
-                      min(lo + 255, hi - 1), min(lo + 256, hi - 1)]
-            last_block = lo + ((hi - lo - 1) // 256) * 256
-            picks += [last_block, max(lo, last_block - 1)]
+                      min(lo + 255, hi - 1), min(lo + 256, hi - 1),
+                      min(lo + 383, hi - 1), min(lo + 384, hi - 1)]
+            for blk in (256, 384):
+                last_block = lo + ((hi - lo - 1) // blk) * blk
+                picks += [last_block, max(lo, last_block - 1)]
     r = raw_u64(stream_key(seed, 40), 0, max(n, 1))
     picks += list((r % np.uint64(max(w.N, 1))).astype(np.int64))
     rows = np.unique(np.asarray(picks, dtype=np.int64))
