@@ -117,64 +117,70 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 
 // Per-row selection state of one thread.  The row's slots live in the warp's block of shared
 // memory in slot-major order (slot s of lane l at [s*32 + l]), so lock-step loops over slots are
-// bank-conflict free.  The k-entry list is unsorted; gmin caches the minimum of each 8-slot group
-// and lmin the minimum of the list (0 = an empty slot, so tau stays -inf until k real entries exist).
+// bank-conflict free.  The k-entry list is unsorted and split into two 32-bit planes: the order-
+// preserving bits of the group maximum (0 = empty slot, ~0 = slot past k) and the group's first
+// key.  gmin caches the minimum of each 8-slot block and lmin the minimum of the list, so tau stays
+// -inf until k real entries exist.  Only the score plane takes part in comparisons: a candidate
+// must beat the list minimum strictly, so of two groups with equal maxima the one met first (the
+// lower keys) stays; among several list entries that tie for the minimum the first slot is replaced.
 template <int KG>
 struct RowSel {
-    cand_t gmin[KG];
-    cand_t lmin;
+    uint32_t gmin[KG];
+    uint32_t lmin;
     float tau;
     int cnt;
 };
 
 template <int KG>
-__device__ __forceinline__ void row_init(RowSel<KG>& r, cand_t* wl, int k, int lane, bool rvalid) {
+__device__ __forceinline__ void row_init(RowSel<KG>& r, uint32_t* wl, int k, int lane, bool rvalid) {
 #pragma unroll 1
-    for (int s = 0; s < 8 * KG; ++s) wl[s * 32 + lane] = (s < k) ? 0ull : ~0ull;  // slots past k are never the minimum
+    for (int s = 0; s < 8 * KG; ++s) wl[s * 32 + lane] = (s < k) ? 0u : ~0u;  // slots past k are never the minimum
 #pragma unroll
-    for (int g = 0; g < KG; ++g) r.gmin[g] = (8 * g < k) ? 0ull : ~0ull;
-    r.lmin = 0ull;
+    for (int g = 0; g < KG; ++g) r.gmin[g] = (8 * g < k) ? 0u : ~0u;
+    r.lmin = 0u;
     r.tau = rvalid ? -CUDART_INF_F : CUDART_INF_F;
     r.cnt = 0;
 }
 
-// All 32 lanes insert their pending candidates into their own lists, in lock step.
+// All 32 lanes insert their pending candidates into their own lists, in lock step.  `wl` is the
+// score plane of the warp's lists, the key plane follows it (8*KG*32 words further).
 template <int KG>
-__device__ __forceinline__ void flush_pending(RowSel<KG>& r, cand_t* wl, const cand_t* wp, int lane, bool rvalid) {
+__device__ __forceinline__ void flush_pending(RowSel<KG>& r, uint32_t* wl, const cand_t* wp, int lane, bool rvalid) {
     const int maxc = __reduce_max_sync(FULL, r.cnt);
     __syncwarp();
 #pragma unroll 1
     for (int t = 0; t < maxc; ++t) {
         if (t < r.cnt) {
             const uint2 raw = *reinterpret_cast<const uint2*>(wp + t * 32 + lane);  // {first key, fp32 bits}
-            const cand_t x = make_cand(__uint_as_float(raw.y), (int)raw.x);
+            const uint32_t x = order_bits(__uint_as_float(raw.y) + 0.0f);
             if (x > r.lmin) {
                 int g = 0;
-                cand_t m = r.gmin[0];
+                uint32_t m = r.gmin[0];
 #pragma unroll
                 for (int q = 1; q < KG; ++q)
                     if (r.gmin[q] < m) { m = r.gmin[q]; g = q; }
-                cand_t* grp = wl + (g * 8) * 32 + lane;
-                cand_t nm = x;
+                uint32_t* grp = wl + (g * 8) * 32 + lane;
+                uint32_t nm = x;
                 int pos = -1;
 #pragma unroll
                 for (int s = 0; s < 8; ++s) {
-                    const cand_t y = grp[s * 32];
-                    if (y == m && pos < 0) pos = s; else nm = cmin(nm, y);
+                    const uint32_t y = grp[s * 32];
+                    if (y == m && pos < 0) pos = s; else nm = min(nm, y);
                 }
                 grp[pos * 32] = x;
+                grp[8 * KG * 32 + pos * 32] = raw.x;
 #pragma unroll
                 for (int q = 0; q < KG; ++q)
                     if (q == g) r.gmin[q] = nm;
-                cand_t lm = r.gmin[0];
+                uint32_t lm = r.gmin[0];
 #pragma unroll
-                for (int q = 1; q < KG; ++q) lm = cmin(lm, r.gmin[q]);
+                for (int q = 1; q < KG; ++q) lm = min(lm, r.gmin[q]);
                 r.lmin = lm;
             }
         }
     }
     r.cnt = 0;
-    if (rvalid) r.tau = r.lmin ? cand_score(r.lmin) : -CUDART_INF_F;
+    if (rvalid) r.tau = r.lmin ? unorder_bits(r.lmin) : -CUDART_INF_F;
 }
 
 // Maxima of the eight 8-column groups of 64 consecutive columns (three-input max; all first-level
@@ -406,8 +412,9 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     } else if (warp < NEPI) {
         // ------------------------------------------------------------------ selection warps
         const int qt = warp >> 2, quarter = warp & 3;
-        cand_t* wl = sRows + (size_t)(qt * 128 + quarter * 32) * Sp::SLOTS;  // this warp's block: list slots ...
-        cand_t* wp = wl + Sp::LIST * 32;                                     // ... then pending slots
+        cand_t* wblock = sRows + (size_t)(qt * 128 + quarter * 32) * Sp::SLOTS;  // this warp's block:
+        uint32_t* wl = reinterpret_cast<uint32_t*>(wblock);                     // the lists (score plane, key plane) ...
+        cand_t* wp = wblock + Sp::LIST * 32;                                    // ... then the pending slots
         const uint32_t wp_addr = ptx::smem_u32(wp + lane);                   // this lane's first pending slot
         RowSel<KG> rs;
         int flush_seen = 0;
@@ -529,9 +536,9 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 for (int r = 0; r < nloc; ++r) {
                     const size_t o = ((size_t)(it.row0 + qt * BM + quarter * 32 + r) * H + h) * k;
                     for (int t = lane; t < k; t += 32) {
-                        const cand_t c = wl[t * 32 + r];
-                        topk_idx[o + t] = c ? cand_index(c) : -1;
-                        topk_score[o + t] = c ? cand_score(c) : -CUDART_INF_F;
+                        const uint32_t c = wl[t * 32 + r];
+                        topk_idx[o + t] = c ? (int)wl[Sp::LIST * 32 + t * 32 + r] : -1;
+                        topk_score[o + t] = c ? unorder_bits(c) : -CUDART_INF_F;
                     }
                 }
                 __syncwarp();
