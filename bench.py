@@ -277,7 +277,7 @@ def run_ours(args, w):
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
-        rows, cores = oracle_rows(w, 16)
+        rows, cores = oracle_rows(w, 64)
         dt_o, sc_o = oracle_step(w, rows)
         result["cpu_baseline"] = {
             "value": sc_o / dt_o, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": dt_o,

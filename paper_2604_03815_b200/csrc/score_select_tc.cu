@@ -2,31 +2,34 @@
 //
 // The paper evaluates S = Q K^T lazily (a "symbolic matrix") on CUDA cores and reduces each row
 // to its k best entries without storing S.  Here the same reduction is fed by the 5th-generation
-// tensor cores: a persistent CTA per SM owns up to 256 query rows (two 128-row tiles) of one
+// tensor cores: a persistent CTA per SM owns up to 384 query rows (NQT 128-row tiles) of one
 // graph and one head, streams that graph's keys in 128-key tiles through a TMA -> shared memory
-// ring, multiplies each tile against both query tiles with tcgen05.mma (bf16 in, fp32
-// accumulators in tensor memory, double buffered), and eight selection warps read the
-// accumulators straight out of tensor memory.  One thread owns one query row.
-//   fast pass   the thread pulls its 128 scores of the tile into registers (the accumulator
-//               buffer goes straight back to the MMA issuer), reduces every 8 consecutive
+// ring, multiplies each key tile against every query tile with tcgen05.mma (bf16 in, fp32
+// accumulators in tensor memory: four 128-column buffers used as a ring by the sequence of
+// (key tile, query tile) pairs), and 4*NQT selection warps read the accumulators straight out of
+// tensor memory.  One thread owns one query row.
+//   fast pass   the thread pulls its 128 scores of the pair into registers (the accumulator
+//               buffer goes straight back to the MMA issuers), reduces every 8 consecutive
 //               columns to their maximum with three-input max instructions and compares the
 //               tile maximum once against the row's threshold tau;
-//   candidates  a candidate is an 8-key GROUP, ranked by its maximum.  The k best groups under
-//               (maximum desc, first key asc) always contain the k best keys under (score desc,
-//               key asc): if a key of the top k sat in a group outside the best k groups, each
-//               of those k groups would hold a key that beats it.  So the sweep only tracks
-//               groups: a lane whose tile maximum beats tau appends (group maximum, first key)
-//               for the groups above tau to its pending slots - no index search, no votes;
-//   flush       when a pending area is half full all 32 lanes insert their pending groups into
-//               their own unsorted k-entry lists in lock step (replace the list minimum, 8-slot
-//               blocks with cached minima) and refresh tau = k-th best group maximum so far.
+//   candidates  a candidate is an 8-key GROUP, ranked by its maximum.  The k groups with the
+//               largest maxima always contain k keys whose scores are the k largest of the row:
+//               if a key of the top k sat in a group outside them, each of the k groups would
+//               hold a key at least as good.  So the sweep only tracks groups: a lane whose tile
+//               maximum beats tau appends (group maximum, first key) for the groups above tau to
+//               its pending slots - no index search.  Groups with EQUAL maxima are not ordered
+//               further (a new one never displaces an equal old one); the rescoring kernel applies
+//               the (score desc, key asc) order to the keys it is given;
+//   flush       when a pending area fills up all 32 lanes insert their pending groups into their
+//               own unsorted k-entry lists in lock step (replace the list minimum, 8-slot blocks
+//               with cached minima) and refresh tau = k-th best group maximum so far.
 // When an item ends each row's k groups go to global memory; refine.cu rescores their 8k keys
 // exactly and keeps the best k.  The N x N scores never leave the SM.
 //
-// Warp roles (NQT = query tiles per CTA, 1 or 2):
-//   warps 0 .. 4*NQT-1   selection; warp w reads TMEM lanes 32*(w%4).. of query tile w/4
+// Warp roles (NQT = query tiles per CTA, 1 to 3):
+//   warps 0 .. 4*NQT-1   selection; warp w reads TMEM lanes 32*(w%4).. for query tile w/4
 //   warp 4*NQT           TMA producer (one lane)
-//   warps 4*NQT+1, +2    tcgen05.mma issue (one lane each, alternating key tiles); +1 owns TMEM
+//   warps 4*NQT+1, +2    tcgen05.mma issue (one lane each, alternating pairs); +1 owns TMEM
 // Every wait is bounded; on expiry the CTA records KMIP_ERR_TIMEOUT, drains and exits normally.
 #include <cuda.h>
 
