@@ -180,22 +180,65 @@ def run_ours(args, w):
                                        fb.topk_idx, fb.topk_score, bb.dQ, bb.dK, bb.dV, bb.workspace)
             assert rc == kb.KMIP_OK, kb.status_string(rc)
 
-    def step_e2e():
-        for n in ("Q", "K", "V", "dOut"):
-            d_in[n].copy_(host[n], non_blocking=True)
-        step()
-        host_out["out"].copy_(fb.out, non_blocking=True)
-        if w.backward:
-            for n in ("dQ", "dK", "dV"):
-                host_out[n].copy_(getattr(bb, n), non_blocking=True)
+    # End-to-end arm: every step copies its inputs from pinned host memory and reads its results
+    # back, through the same two public calls.  Two sets of device buffers let the copies of one
+    # step overlap the kernels of its neighbours (inputs of step i+1 arrive and results of step
+    # i-1 leave while step i computes), ordered by events; all of it is inside the timed region.
+    e2e = None
 
-    def timed(fn, steps):
+    def e2e_setup():
+        sets = []
+        for s_ in range(2):
+            sets.append({
+                "in": {n: torch.empty_like(d_in[n]) for n in d_in},
+                "fb": kb.ForwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode, dev),
+                "bb": kb.BackwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode, dev),
+                "h2d": torch.cuda.Event(), "comp": torch.cuda.Event(), "d2h": torch.cuda.Event(),
+            })
+            sets[-1]["comp"].record()
+            sets[-1]["d2h"].record()
+        return {"sets": sets, "s_in": torch.cuda.Stream(dev), "s_out": torch.cuda.Stream(dev), "i": 0}
+
+    def step_e2e():
+        cur = torch.cuda.current_stream()
+        st = e2e["sets"][e2e["i"] % 2]
+        e2e["i"] += 1
+        with torch.cuda.stream(e2e["s_in"]):
+            e2e["s_in"].wait_event(st["comp"])          # the step that last read this set has finished
+            for n in ("Q", "K", "V", "dOut"):
+                st["in"][n].copy_(host[n], non_blocking=True)
+            st["h2d"].record()
+        cur.wait_event(st["h2d"])
+        cur.wait_event(st["d2h"])                        # this set's previous results have left the device
+        rc = kb.kmip_attn_forward(st["in"]["Q"], st["in"]["K"], st["in"]["V"], offs, w.k, w.mode, st["fb"].out,
+                                  st["fb"].topk_idx, st["fb"].topk_score, st["fb"].workspace)
+        assert rc == kb.KMIP_OK, kb.status_string(rc)
+        if w.backward:
+            rc = kb.kmip_attn_backward(st["in"]["Q"], st["in"]["K"], st["in"]["V"], offs, w.k, w.mode, st["fb"].out,
+                                       st["in"]["dOut"], st["fb"].topk_idx, st["fb"].topk_score, st["bb"].dQ,
+                                       st["bb"].dK, st["bb"].dV, st["bb"].workspace)
+            assert rc == kb.KMIP_OK, kb.status_string(rc)
+        st["comp"].record()
+        with torch.cuda.stream(e2e["s_out"]):
+            e2e["s_out"].wait_event(st["comp"])
+            host_out["out"].copy_(st["fb"].out, non_blocking=True)
+            if w.backward:
+                for n in ("dQ", "dK", "dV"):
+                    host_out[n].copy_(getattr(st["bb"], n), non_blocking=True)
+            st["d2h"].record()
+
+    def e2e_drain():
+        torch.cuda.current_stream().wait_stream(e2e["s_out"])   # the last results are on the host before the clock stops
+
+    def timed(fn, steps, drain=None):
         kdist.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
             fn()
+        if drain is not None:
+            drain()
         e1.record()
         torch.cuda.synchronize()
         kdist.barrier()
@@ -215,9 +258,13 @@ def run_ours(args, w):
     kb.kmip_profile_enable(0)
     assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
 
+    e2e = e2e_setup()
     for _ in range(min(args.warmup, 2)):
         step_e2e()
-    secs_e2e = timed(step_e2e, args.steps)
+    e2e_drain()
+    secs_e2e = timed(step_e2e, args.steps, e2e_drain)
+    for st_ in e2e["sets"]:
+        assert kb.kmip_last_status(st_["fb"].workspace) == kb.KMIP_OK and kb.kmip_last_status(st_["bb"].workspace) == kb.KMIP_OK
 
     units = float(w.n_scores) * args.steps
     value, t_max = kdist.aggregate_throughput(units, secs)
@@ -270,6 +317,7 @@ def run_ours(args, w):
             "peak_gbs": peaks["hbm_gbs"],
         },
         "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": 1e3 * secs_e2e / args.steps,
+                "overlap": "two device buffer sets: a step's copies overlap its neighbours' kernels, all inside the timed region",
                 "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host.values())),
                 "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for n, t in host_out.items()
                                               if w.backward or n == "out"))},
