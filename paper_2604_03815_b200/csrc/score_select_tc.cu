@@ -145,16 +145,18 @@ __device__ __forceinline__ void row_init(RowSel<KG>& r, uint32_t* wl, int k, int
     r.cnt = 0;
 }
 
-// All 32 lanes insert their pending candidates into their own lists, in lock step.  `wl` is the
-// score plane of the warp's lists, the key plane follows it (8*KG*32 words further).
+// All 32 lanes insert their pending candidates into their own lists, in lock step.  `wl_s` is the
+// shared address of the lane's slot 0 in the score plane of the warp's lists (slots 128 bytes
+// apart, the key plane 8*KG*128 bytes further), `wp_s` that of the lane's first pending slot
+// (256 bytes apart).
 template <int KG>
-__device__ __forceinline__ void flush_pending(RowSel<KG>& r, uint32_t* wl, const cand_t* wp, int lane, bool rvalid) {
+__device__ __forceinline__ void flush_pending(RowSel<KG>& r, uint32_t wl_s, uint32_t wp_s, bool rvalid) {
     const int maxc = __reduce_max_sync(FULL, r.cnt);
     __syncwarp();
 #pragma unroll 1
     for (int t = 0; t < maxc; ++t) {
         if (t < r.cnt) {
-            const uint2 raw = *reinterpret_cast<const uint2*>(wp + t * 32 + lane);  // {first key, fp32 bits}
+            const uint2 raw = ptx::lds_v2(wp_s + (uint32_t)t * 256u);  // {first key, fp32 bits}
             const uint32_t x = order_bits(__uint_as_float(raw.y) + 0.0f);
             if (x > r.lmin) {
                 int g = 0;
@@ -162,16 +164,16 @@ __device__ __forceinline__ void flush_pending(RowSel<KG>& r, uint32_t* wl, const
 #pragma unroll
                 for (int q = 1; q < KG; ++q)
                     if (r.gmin[q] < m) { m = r.gmin[q]; g = q; }
-                uint32_t* grp = wl + (g * 8) * 32 + lane;
+                const uint32_t grp = wl_s + (uint32_t)g * (8u * 128u);
                 uint32_t nm = x;
                 int pos = -1;
 #pragma unroll
                 for (int s = 0; s < 8; ++s) {
-                    const uint32_t y = grp[s * 32];
+                    const uint32_t y = ptx::lds_u32(grp + s * 128);
                     if (y == m && pos < 0) pos = s; else nm = min(nm, y);
                 }
-                grp[pos * 32] = x;
-                grp[8 * KG * 32 + pos * 32] = raw.x;
+                ptx::sts_u32(grp + (uint32_t)pos * 128u, x);
+                ptx::sts_u32(grp + (uint32_t)pos * 128u + 8u * KG * 128u, raw.x);
 #pragma unroll
                 for (int q = 0; q < KG; ++q)
                     if (q == g) r.gmin[q] = nm;
@@ -418,7 +420,10 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         cand_t* wblock = sRows + (size_t)(qt * 128 + quarter * 32) * Sp::SLOTS;  // this warp's block:
         uint32_t* wl = reinterpret_cast<uint32_t*>(wblock);                     // the lists (score plane, key plane) ...
         cand_t* wp = wblock + Sp::LIST * 32;                                    // ... then the pending slots
-        const uint32_t wp_addr = ptx::smem_u32(wp + lane);                   // this lane's first pending slot
+        const uint32_t wp_addr = ptx::smem_u32(wp + lane);                      // this lane's first pending slot
+        const uint32_t wl_s = ptx::smem_u32(wl + lane);                         // this lane's list slot 0 (score plane)
+        const uint32_t flush_req_s = ptx::smem_u32(const_cast<int*>(sFlushReq));
+        const uint32_t full_bar0 = bars.t_full(0, qt);
         RowSel<KG> rs;
         int flush_seen = 0;
         int tcnt = 0;
@@ -436,14 +441,19 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             __syncwarp();
             const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
             for (int j = 0; j < ntiles; ++j, ++tcnt) {
-                const int seq = tcnt * NQT + qt;  // this warp group's (key tile, query tile) pair
-                const int b = seq & (NBUF - 1);
+                // this warp group's (key tile, query tile) pair is number tcnt*NQT + qt of the CTA; its
+                // buffer is that number mod 4, and the (buffer, query tile) barrier has been used
+                // tcnt >> kUseShift times before (pairs between two uses: 12, 4, 4 for NQT = 3, 2, 1)
+                constexpr int kUseShift = NQT == 2 ? 1 : 2;
+                const int b = (tcnt * NQT + qt) & (NBUF - 1);
+                const uint32_t full_bar = full_bar0 + (uint32_t)b * (8u * NQT);
+                const uint32_t full_par = (uint32_t)(tcnt >> kUseShift) & 1u;
                 const long long c0 = (dbg & 8) ? clock64() : 0;
-                if (!__all_sync(FULL, ptx::mbar_try_wait(bars.t_full(b, qt), (seq / Sp::PERIOD) & 1))) {
+                if (!__all_sync(FULL, ptx::mbar_try_wait(full_bar, full_par))) {
                     // The scores are not ready yet: use the wait to merge pending candidates into the
                     // lists (always allowed, and it raises the thresholds early), then block.
-                    if (!DUMP && active && !(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) flush_pending<KG>(rs, wl, wp, lane, rvalid);
-                    ok = wait_or_abort(bars.t_full(b, qt), (seq / Sp::PERIOD) & 1, sAbort, sb, 6, wait_limit);
+                    if (!DUMP && active && !(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
+                    ok = wait_or_abort(full_bar, full_par, sAbort, sb, 6, wait_limit);
                     ok = __all_sync(FULL, ok);
                     if (!ok) break;
                 }
@@ -502,7 +512,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                             // A flush by one warp stalls the other seven within two tiles (the accumulator
                             // buffers are only two deep), so the warps flush together: whoever must flush
                             // bumps a CTA-wide counter and every warp that sees it move flushes at its next tile.
-                            const int req = *sFlushReq;
+                            const int req = (int)ptx::lds_u32(flush_req_s);
                             bool do_flush = req != flush_seen;
                             if (__any_sync(FULL, gm > rs.tau)) {  // some lane of the warp has a hit in this tile
                                 uint32_t pend = wp_addr + (uint32_t)rs.cnt * 256u;
@@ -516,7 +526,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                             }
                             if (do_flush) {
                                 const long long p1 = (dbg & 8) ? clock64() : 0;
-                                flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                                flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
                                 flush_seen = req + ((req == flush_seen) ? 1 : 0);
                                 if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
                             }
@@ -533,7 +543,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (!DUMP && active) {
                 // finalise: drain the pending slots, then store each row's k groups (first key and
                 // group maximum, unsorted; empty slots as -1 / -inf) for the rescoring kernel
-                flush_pending<KG>(rs, wl, wp, lane, rvalid);
+                flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
                 __syncwarp();
                 const int nloc = min(32, it.nrows - (qt * BM + quarter * 32));
                 for (int r = 0; r < nloc; ++r) {
