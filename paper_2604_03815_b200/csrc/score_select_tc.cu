@@ -92,7 +92,6 @@ struct SmemPlan {
     static constexpr int LIST = 8 * KG;               // list slots per row (k <= LIST)
     static constexpr int ROOM = NQT >= 3 ? 24 : 32;   // pending candidate slots per row (a tile adds at most 16)
     static constexpr int SLOTS = LIST + ROOM;         // cand_t per row
-    static constexpr int PERIOD = NQT == 3 ? 12 : 4;  // pairs between two uses of a buffer by the same query tile
     static constexpr int NBARS = 3 + 2 * S + NBUF * NQT + NBUF;
 };
 
