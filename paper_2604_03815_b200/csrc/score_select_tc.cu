@@ -423,13 +423,13 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t wl_s = ptx::smem_u32(wl + lane);                         // this lane's list slot 0 (score plane)
         const uint32_t flush_req_s = ptx::smem_u32(const_cast<int*>(sFlushReq));
         const uint32_t full_bar0 = bars.t_full(0, qt);
+        const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16);  // buffer 0, this warp's lanes
         RowSel<KG> rs;
         int flush_seen = 0;
         int tcnt = 0;
         bool ok = true;
         long long w_tfull = 0, t_work = 0, t_begin = clock64();
         long long prof[4] = {0, 0, 0, 0};
-        long long ph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
             const int h = (int)(w / n_items);
             const WorkItem it = items[w % n_items];
@@ -439,78 +439,87 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (active) row_init<KG>(rs, wl, k, lane, rvalid);
             __syncwarp();
             const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
-            for (int j = 0; j < ntiles; ++j, ++tcnt) {
-                // this warp group's (key tile, query tile) pair is number tcnt*NQT + qt of the CTA; its
-                // buffer is that number mod 4, and the (buffer, query tile) barrier has been used
-                // tcnt >> kUseShift times before (pairs between two uses: 12, 4, 4 for NQT = 3, 2, 1)
-                constexpr int kUseShift = NQT == 2 ? 1 : 2;
-                const int b = (tcnt * NQT + qt) & (NBUF - 1);
-                const uint32_t full_bar = full_bar0 + (uint32_t)b * (8u * NQT);
-                const uint32_t full_par = (uint32_t)(tcnt >> kUseShift) & 1u;
-                const long long c0 = (dbg & 8) ? clock64() : 0;
-                if (!__all_sync(FULL, ptx::mbar_try_wait(full_bar, full_par))) {
-                    // The scores are not ready yet: use the wait to merge pending candidates into the
-                    // lists (always allowed, and it raises the thresholds early), then block.
-                    if (!DUMP && active && !(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
-                    ok = wait_or_abort(full_bar, full_par, sAbort, sb, 6, wait_limit);
+            // This warp group's (key tile, query tile) pair is number tcnt*NQT + qt of the CTA; its buffer
+            // is that number mod 4, and the (buffer, query tile) barrier has been used tcnt >> kUseShift
+            // times before (pairs between two uses: 12, 4, 4 for NQT = 3, 2, 1).
+            constexpr int kUseShift = NQT == 2 ? 1 : 2;
+            if (DUMP || !active) {
+                // debug dump of the raw scores, or a query tile past the item's rows that only keeps
+                // the barriers in step
+                for (int j = 0; j < ntiles; ++j, ++tcnt) {
+                    const int b = (tcnt * NQT + qt) & (NBUF - 1);
+                    ok = wait_or_abort(full_bar0 + (uint32_t)b * (8u * NQT), (uint32_t)(tcnt >> kUseShift) & 1u, sAbort, sb,
+                                       6, wait_limit);
                     ok = __all_sync(FULL, ok);
                     if (!ok) break;
-                }
-                const long long c1 = (dbg & 8) ? clock64() : 0;
-                // this query tile's MMAs on the key tile have retired; once that holds for every query
-                // tile the key stage can be refilled
-                if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
-                ptx::tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * BN);
-                const int key0 = it.key_lo + j * BN;
-                const int ncol = min(BN, it.key_hi - key0);
-                if (DUMP) {
+                    if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
+                    ptx::tc_fence_after();
+                    if (DUMP && active) {
+                        const uint32_t taddr = taddr0 + (uint32_t)(b * BN);
+                        const int key0 = it.key_lo + j * BN;
+                        const int ncol = min(BN, it.key_hi - key0);
 #pragma unroll 1
-                    for (int c = 0; c < BN / 32; ++c) {
-                        uint32_t v[32];
-                        ptx::tmem_ld_32x32_sync(taddr + c * 32, v);
-                        if (active && rvalid)
+                        for (int c = 0; c < BN / 32; ++c) {
+                            uint32_t v[32];
+                            ptx::tmem_ld_32x32_sync(taddr + c * 32, v);
+                            if (rvalid)
 #pragma unroll
-                            for (int x = 0; x < 32; ++x)
-                                if (c * 32 + x < ncol)
-                                    dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + c * 32 + x] = __uint_as_float(v[x]);
+                                for (int x = 0; x < 32; ++x)
+                                    if (c * 32 + x < ncol)
+                                        dump[((size_t)h * dump_ld + it.row0 + local) * dump_ld + key0 + c * 32 + x] = __uint_as_float(v[x]);
+                        }
                     }
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
-                } else {
+                }
+            } else {
+                const int ragged_j = ((it.key_hi - it.key_lo) & (BN - 1)) ? ntiles - 1 : -1;  // only the last tile can be short
+                int key0 = it.key_lo;
+                for (int j = 0; j < ntiles; ++j, ++tcnt, key0 += BN) {
+                    const int b = (tcnt * NQT + qt) & (NBUF - 1);
+                    const uint32_t full_bar = full_bar0 + (uint32_t)b * (8u * NQT);
+                    const uint32_t full_par = (uint32_t)(tcnt >> kUseShift) & 1u;
+                    const long long c0 = (dbg & 8) ? clock64() : 0;
+                    if (!__all_sync(FULL, ptx::mbar_try_wait(full_bar, full_par))) {
+                        // The scores are still not there after the try's own (hardware-bounded) wait:
+                        // merge pending candidates into the lists meanwhile (always allowed, and it
+                        // raises the thresholds early), then block.
+                        if (!(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
+                        ok = wait_or_abort(full_bar, full_par, sAbort, sb, 6, wait_limit);
+                        ok = __all_sync(FULL, ok);
+                        if (!ok) break;
+                    }
+                    const long long c1 = (dbg & 8) ? clock64() : 0;
+                    // this query tile's MMAs on the key tile have retired; once that holds for every query
+                    // tile the key stage can be refilled
+                    if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
+                    ptx::tc_fence_after();
+                    const uint32_t taddr = taddr0 + (uint32_t)(b * BN);
+                    const bool ragged = j == ragged_j;
+                    const int ncol = it.key_hi - key0;  // columns that exist; below 128 only in a ragged tile
                     // two 64-column halves keep the register footprint small; the accumulator buffer
-                    // goes back to the MMA issuer as soon as the second half is in registers
+                    // goes back to the MMA issuers as soon as the second half is in registers
                     float sub[16], quad[4];
                     uint32_t v[64];
-                    const bool ragged = ncol < BN;
-                    long long s0 = 0, s1 = 0, s2 = 0, s3 = 0, s4 = 0;
-                    if (dbg & 32) s0 = clock64();
-                    if (active) {
-                        ptx::tmem_ld_32x64_sync(taddr, v);
-                        if (dbg & 32) s1 = clock64();
-                        if (!(dbg & 2)) {
-                            if (ragged) half_maxima<true>(v, ncol, sub, quad);
-                            else half_maxima<false>(v, ncol, sub, quad);
-                        }
-                        if (dbg & 32) s2 = clock64();
-                        ptx::tmem_ld_32x64_sync(taddr + 64, v);
-                        if (dbg & 32) s3 = clock64();
+                    ptx::tmem_ld_32x64_sync(taddr, v);
+                    if (!(dbg & 2)) {
+                        if (ragged) half_maxima<true>(v, ncol, sub, quad);
+                        else half_maxima<false>(v, BN, sub, quad);
                     }
+                    ptx::tmem_ld_32x64_sync(taddr + 64, v);
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
-                    if (dbg & 32) { s4 = clock64(); ph[0] += s0 - c1; ph[1] += s1 - s0; ph[2] += s2 - s1; ph[3] += s3 - s2; ph[4] += s4 - s3; }
-                    if (active && !(dbg & 2)) {
+                    if (!(dbg & 2)) {
                         if (ragged) half_maxima<true>(v, ncol - 64, sub + 8, quad + 2);
-                        else half_maxima<false>(v, ncol - 64, sub + 8, quad + 2);
+                        else half_maxima<false>(v, BN, sub + 8, quad + 2);
                         const float gm = fmaxf(fmaxf(quad[0], quad[1]), fmaxf(quad[2], quad[3]));
-                        if (dbg & 32) { if (gm == 77.125f) rs.tau = 1.0f; ph[5] += clock64() - s4; }
                         if (!(dbg & 1)) {
                             const long long p0 = (dbg & 8) ? clock64() : 0;
-                            // A flush by one warp stalls the other seven within two tiles (the accumulator
-                            // buffers are only two deep), so the warps flush together: whoever must flush
-                            // bumps a CTA-wide counter and every warp that sees it move flushes at its next tile.
+                            // A flush by one warp stalls the others within a few tiles (the accumulator ring
+                            // is only four deep), so the warps flush together: whoever must flush bumps a
+                            // CTA-wide counter and every warp that sees it move flushes at its next tile.
                             const int req = (int)ptx::lds_u32(flush_req_s);
                             bool do_flush = req != flush_seen;
                             if (__any_sync(FULL, gm > rs.tau)) {  // some lane of the warp has a hit in this tile
@@ -532,11 +541,11 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         } else if (gm == 123.456f) {
                             rs.tau = 0.0f;  // timing experiment: keep the maxima alive
                         }
-                    } else if (active && v[0] == 0x12345678u && v[63] == 1u) {
+                    } else if (v[0] == 0x12345678u && v[63] == 1u) {
                         rs.tau = 0.0f;  // timing experiment: keep the loads alive
                     }
+                    if (dbg & 8) { w_tfull += c1 - c0; t_work += clock64() - c1; }
                 }
-                if (dbg & 8) { w_tfull += c1 - c0; t_work += clock64() - c1; }
             }
             if (!ok) break;
             if (!DUMP && active) {
@@ -562,7 +571,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             timing[blockIdx.x * 8 + 6] = t_work;
             timing[blockIdx.x * 8 + 7] = tcnt;
             for (int i = 0; i < 4; ++i) timing[148 * 8 + blockIdx.x * 8 + i] = prof[i];
-            for (int i = 0; i < 8; ++i) timing[148 * 16 + blockIdx.x * 8 + i] = ph[i];
         }
     }
 
