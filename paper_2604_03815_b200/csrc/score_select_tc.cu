@@ -90,7 +90,7 @@ constexpr int NBUF = 4;  // accumulator buffers of BN columns: all 512 columns o
 template <int KG, int NQT, int S>
 struct SmemPlan {
     static constexpr int LIST = 8 * KG;               // list slots per row (k <= LIST)
-    static constexpr int ROOM = NQT >= 3 ? 24 : 32;   // pending candidate slots per row (a tile adds at most 16)
+    static constexpr int ROOM = (NQT >= 3 || (NQT == 2 && KG >= 8)) ? 24 : 32;  // pending candidate slots per row (a tile adds at most 16)
     static constexpr int SLOTS = LIST + ROOM;         // cand_t per row
     static constexpr int NBARS = 3 + 2 * S + NBUF * NQT + NBUF;
 };
@@ -667,7 +667,8 @@ cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
         else return launch_cfg<D, 4, 1, 3, DUMP>(a, w, dump);
     }
     if (a.k <= 64) {
-        if constexpr (D <= 64) return launch_cfg<D, 8, 1, 4, DUMP>(a, w, dump);
+        if constexpr (D <= 32) return launch_cfg<D, 8, 2, 3, DUMP>(a, w, dump);
+        else if constexpr (D == 64) return launch_cfg<D, 8, 1, 4, DUMP>(a, w, dump);
         else return launch_cfg<D, 8, 1, 3, DUMP>(a, w, dump);
     }
     if constexpr (D <= 64) return launch_cfg<D, 16, 1, 3, DUMP>(a, w, dump);
@@ -705,7 +706,10 @@ bool score_select_tc_supported(int32_t d, int32_t k) {
     return k <= 128 && d <= 64;
 }
 
-int score_select_tc_rows_per_item(int32_t d, int32_t k) { return k > 32 || d > 64 ? 128 : d > 32 ? 256 : 384; }  // 128 * query tiles per CTA
+int score_select_tc_rows_per_item(int32_t d, int32_t k) {  // 128 * query tiles per CTA of launch_d's choice
+    if (k <= 32) return d <= 32 ? 384 : d == 64 ? 256 : 128;
+    return (k <= 64 && d <= 32) ? 256 : 128;
+}  // 128 * query tiles per CTA
 
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w) {
     return launch_any<false>(a, w, nullptr);
