@@ -142,6 +142,18 @@ def iid_workload(name, seed, sizes, H, d, k, mode, input_scale=1.0, backward=Tru
     )
 
 
+def padded_workload(name, seed, N, H, d_model, d_pad, k, mode, backward=True) -> Workload:
+    """One graph of N nodes with d_model-wide heads stored zero-padded to d_pad columns (the
+    library takes head widths 16, 32, 64, 128; zero columns leave every inner product and every
+    output column of the first d_model unchanged).  The softmax scale follows the stored width,
+    so a caller who wants 1/sqrt(d_model) multiplies Q by sqrt(d_pad / d_model) first."""
+    w = iid_workload(name, seed, [N], H, d_pad, k, mode, backward=backward)
+    for a in (w.Q, w.K, w.V, w.dOut):
+        a[:, :, d_model:] = 0.0
+    w.meta["d_model"] = d_model
+    return w
+
+
 def config1() -> Workload:
     """One graph, N=1024, H=1, d=32, k=16, fp32 exact mode, values N(0,1)/sqrt(d), seed 0."""
     return iid_workload("c1_single_1k_fp32", 0, [1024], 1, 32, 16, MODE_FP32_EXACT,

@@ -103,6 +103,14 @@ def test_item_and_ring_boundaries():
         assert st["rows"] == sum(sizes)
 
 
+@pytest.mark.parametrize("mode", [wl.MODE_BF16_TC, wl.MODE_FP32_EXACT])
+def test_padded_head_width_of_the_paper_sweep(mode):
+    """d_K = 10 stored zero-padded to 16 columns, k = 10, one head (the shape of the paper's size
+    sweep): same parity bar as every other shape, and the padded output and gradient columns stay zero."""
+    w = wl.padded_workload("s", 91, 3000, 1, 10, 16, 10, mode)
+    _fwd_bwd(w)
+
+
 def test_single_node():
     w = wl.iid_workload("s", 78, [1], 2, 16, 4, wl.MODE_BF16_TC)
     dev = pu.to_device(w)
