@@ -82,11 +82,15 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
     if (tc && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
-    if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 256) != cudaSuccess) return KMIP_ERR_CUDA;
+    const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k);
+    if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
-    if ((tc ? launch_score_select_tc(a, w) : launch_score_select_exact(a)) != cudaSuccess) return KMIP_ERR_CUDA;
+    const cudaError_t sweep = tc ? launch_score_select_tc(a, w)
+                              : tiled32 ? launch_score_select_fp32_tiled(a, w) : launch_score_select_exact(a);
+    if (sweep != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], a.stream);
     if (tc && launch_refine_topk(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (tiled32 && launch_refine_topk_fp32(a) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[3], a.stream);
     if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4], a.stream);

@@ -28,14 +28,16 @@ __device__ inline int graph_end(const int32_t* offs, int G, int N, int i) {
     return max(0, min(N, __ldg(offs + a + 1)));
 }
 
-template <typename T, int D, int E>
+// REGROUPED: `Kp` is the bf16 copy of K regrouped by head, [H, N, D] (tensor-core mode); otherwise it is
+// K itself, [N, H, D] (fp32 mode, scores by fp32 FMA in index order as in the exact kernel).
+template <typename T, int D, int E, bool REGROUPED>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int32_t* __restrict__ offs, int G,
                    int N, int H, int k, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
                    const StatusBlock* __restrict__ sb) {
     if (sb->status != KMIP_OK) return;
     constexpr int CAP = 32 * E;
-    static_assert(sizeof(T) == 2, "the rescoring kernel reads bf16 keys");
+    static_assert((sizeof(T) == 2) == REGROUPED, "bf16 keys come regrouped, fp32 keys in place");
     __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
     __shared__ float s_q[kWarpsPerBlock][D];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -92,8 +94,9 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                 jj[u] = g + (lane % kGroup);
                 valid[u] = t < k && g >= 0 && jj[u] < hi;
                 if (valid[u]) {
-                    // keys regrouped by head: the 8 keys of a group are 8 consecutive rows
-                    const uint4* kr = reinterpret_cast<const uint4*>(Kp + ((size_t)h * N + jj[u]) * D);
+                    // regrouped by head, the 8 keys of a group are 8 consecutive rows
+                    const uint4* kr = reinterpret_cast<const uint4*>(
+                        REGROUPED ? Kp + ((size_t)h * N + jj[u]) * D : Kp + ((size_t)jj[u] * H + h) * D);
 #pragma unroll
                     for (int v = 0; v < NV; ++v) raw[u][v] = __ldg(kr + v);
                 }
@@ -107,8 +110,12 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                         const uint32_t wv[4] = {raw[u][v].x, raw[u][v].y, raw[u][v].z, raw[u][v].w};
 #pragma unroll
                         for (int x = 0; x < 4; ++x) {
-                            s = fmaf(q[v * 8 + 2 * x], __uint_as_float(wv[x] << 16), s);
-                            s = fmaf(q[v * 8 + 2 * x + 1], __uint_as_float(wv[x] & 0xFFFF0000u), s);
+                            if constexpr (sizeof(T) == 2) {
+                                s = fmaf(q[v * 8 + 2 * x], __uint_as_float(wv[x] << 16), s);
+                                s = fmaf(q[v * 8 + 2 * x + 1], __uint_as_float(wv[x] & 0xFFFF0000u), s);
+                            } else {
+                                s = fmaf(q[v * 4 + x], __uint_as_float(wv[x]), s);
+                            }
                         }
                     }
                 }
@@ -129,14 +136,14 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
     }
 }
 
-template <int D>
-cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w) {
-    using T = __nv_bfloat16;
+template <typename T, int D>
+cudaError_t launch_d(const FwdArgs& a, const T* keys) {
+    constexpr bool REGROUPED = sizeof(T) == 2;
     const long long n_rows = (long long)a.N * a.H;
     const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
 #define KMIP_LAUNCH_REFINE(E_) \
-    refine_topk_kernel<T, D, E_><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
-        static_cast<const T*>(a.Q), reinterpret_cast<const T*>(a.ws + w.kpack_off), a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
+    refine_topk_kernel<T, D, E_, REGROUPED><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
+        static_cast<const T*>(a.Q), keys, a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
         a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws))
     // pending room CAP-k >= 96, so that the survivors of a row (rarely more than 2k) fit without
     // intermediate compactions
@@ -149,11 +156,24 @@ cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w) {
 }  // namespace
 
 cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w) {
+    using T = __nv_bfloat16;
+    const T* keys = reinterpret_cast<const T*>(a.ws + w.kpack_off);
     switch (a.d) {
-        case 16: return launch_d<16>(a, w);
-        case 32: return launch_d<32>(a, w);
-        case 64: return launch_d<64>(a, w);
-        case 128: return launch_d<128>(a, w);
+        case 16: return launch_d<T, 16>(a, keys);
+        case 32: return launch_d<T, 32>(a, keys);
+        case 64: return launch_d<T, 64>(a, keys);
+        case 128: return launch_d<T, 128>(a, keys);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+// fp32 mode (tiled CUDA-core sweep): the keys are read in place.
+cudaError_t launch_refine_topk_fp32(const FwdArgs& a) {
+    const float* keys = static_cast<const float*>(a.K);
+    switch (a.d) {
+        case 16: return launch_d<float, 16>(a, keys);
+        case 32: return launch_d<float, 32>(a, keys);
+        case 64: return launch_d<float, 64>(a, keys);
         default: return cudaErrorInvalidValue;
     }
 }
