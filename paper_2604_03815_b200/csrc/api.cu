@@ -28,6 +28,7 @@ struct Profile {
     cudaEvent_t bwd[kProfMaxCalls][4];
 };
 Profile g_prof;
+int g_fp32_path = 0;  // test hook, see kmip_debug_fp32_path
 
 }  // namespace
 
@@ -82,7 +83,10 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
     if (tc && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
-    const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k);
+    // the tiled fp32 sweep runs one block per 128 query rows and head: worth it once that fills the GPU
+    // about twice, below that the one-warp-per-row kernel has more parallelism
+    const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k) &&
+                         (g_fp32_path == 0 ? (N / 128) * H >= 296 : g_fp32_path == 2);
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
     const cudaError_t sweep = tc ? launch_score_select_tc(a, w)
@@ -175,6 +179,10 @@ int kmip_profile_read(double* stage_ms, int* calls) {
     g_prof.n_fwd = g_prof.n_bwd = 0;
     return KMIP_OK;
 }
+
+// ---- test hook (not part of kmip.h): which fp32-mode sweep runs; 0 = by problem size, 1 = always one
+// warp per row, 2 = the tiled sweep whenever it supports (d, k), so that tests can put both on the same inputs
+void kmip_debug_fp32_path(int which) { g_fp32_path = which; }
 
 // ---- timing experiments (not part of kmip.h): see set_score_select_debug_flags
 void kmip_debug_set_flags(int flags) { set_score_select_debug_flags(flags); }

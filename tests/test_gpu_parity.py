@@ -132,6 +132,52 @@ def test_identical_keys_tie_break_by_index(mode):
     pu.check_forward(w, fb)
 
 
+# fp32 problems with at least 296 blocks of 128 rows x heads run the tiled CUDA-core sweep and the
+# fp32 rescoring kernel instead of the one-warp-per-row kernel the small fp32 cases above exercise
+@pytest.mark.parametrize("d,k", [(16, 10), (32, 32), (64, 17)])
+def test_fp32_tiled_sweep(d, k):
+    sizes = [3000, 129, 5000, 1, 2000, 383, 0, 64]
+    w = wl.iid_workload("s", 3000 + d, sizes, 4, d, k, wl.MODE_FP32_EXACT, input_scale=1.0 / np.sqrt(d))
+    assert (w.N // 128) * w.H >= 296
+    st = _fwd_bwd(w)
+    assert st["identical_rows"] > 0.999   # all but rows where two neighbouring scores tie within fp32 rounding
+
+
+def test_fp32_tiled_sweep_tie_break_by_index():
+    """Identical keys inside each graph: every score of a row ties, so the answer is the k lowest
+    key indices of the graph, and equal group maxima must be ordered by their first key."""
+    w = wl.iid_workload("s", 3100, [6000, 4500], 4, 16, 12, wl.MODE_FP32_EXACT)
+    w.K[:] = w.K[7]
+    assert (w.N // 128) * w.H >= 296
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    idx = fb.topk_idx.cpu().numpy()
+    assert np.all(idx[:6000] == np.arange(12)) and np.all(idx[6000:] == 6000 + np.arange(12))
+    pu.check_forward(w, fb)
+
+
+@pytest.mark.parametrize("d,k", [(16, 5), (32, 16), (64, 32)])
+def test_fp32_sweeps_agree_bit_for_bit(d, k):
+    """The two fp32-mode sweeps (one warp per row; tiled, thread per row) run the same fp32 FMAs in
+    the same order and the same (score desc, key asc) rule: identical outputs on ragged batches
+    with tiny and empty graphs, whichever the library would pick by size."""
+    sizes = [1, 0, 3, 129, 0, 7, 256, 2, 385, 16, 31, 33, 700]
+    w = wl.iid_workload("s", 3200 + d, sizes, 2, d, k, wl.MODE_FP32_EXACT, input_scale=1.0 / np.sqrt(d))
+    dev = pu.to_device(w)
+    res = []
+    try:
+        for path in (1, 2):
+            kb.lib().kmip_debug_fp32_path(path)
+            fb = pu.run_forward(w, dev)
+            torch.cuda.synchronize()
+            res.append((fb.topk_idx.cpu().numpy().copy(), fb.topk_score.cpu().numpy().copy(), fb.out.cpu().numpy().copy()))
+    finally:
+        kb.lib().kmip_debug_fp32_path(0)
+    for a, b in zip(res[0], res[1]):
+        assert np.array_equal(a, b)
+    pu.check_forward(w, fb)
+
+
 def test_null_offsets_means_one_graph():
     w = wl.iid_workload("s", 80, [600], 2, 32, 8, wl.MODE_BF16_TC)
     Q, K, V, dO, offs = pu.to_device(w)
