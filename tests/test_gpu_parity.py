@@ -228,6 +228,45 @@ def test_bounded_wait_runs_out_and_is_reported():
     pu.check_forward(w, pu.run_forward(w, dev))
 
 
+def test_forward_and_backward_replay_from_a_cuda_graph():
+    """Both calls only enqueue work on the caller's stream (no allocation, no synchronisation), so a
+    forward + backward pair can be captured once and replayed on new input values."""
+    w = wl.make_config(2)
+    Q, K, V, dO, offs = pu.to_device(w)
+    G = len(w.graph_offsets) - 1
+    fb = kb.ForwardBuffers(w.N, G, w.H, w.d, w.k, w.mode)
+    bb = kb.BackwardBuffers(w.N, G, w.H, w.d, w.k, w.mode)
+
+    def step():
+        assert kb.kmip_attn_forward(Q, K, V, offs, w.k, w.mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace) == kb.KMIP_OK
+        assert kb.kmip_attn_backward(Q, K, V, offs, w.k, w.mode, fb.out, dO, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK,
+                                     bb.dV, bb.workspace) == kb.KMIP_OK
+
+    step()  # first call outside the capture (driver entry points, kernel attributes)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    # new values in the same buffers: rows reversed inside the batch would change graphs, so scale instead
+    Q.mul_(-1.0)
+    dO.mul_(0.5)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
+    got = [t.clone() for t in (fb.out, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK, bb.dV)]
+    step()  # eager, same inputs
+    torch.cuda.synchronize()
+    for a, b in zip(got[:3], (fb.out, fb.topk_idx, fb.topk_score)):
+        assert torch.equal(a, b)
+    for a, b in zip(got[3:], (bb.dQ, bb.dK, bb.dV)):   # hit lists are filled with atomics: equal up to summation order
+        assert torch.allclose(a.float(), b.float(), rtol=2e-2, atol=2e-3)
+    w2 = wl.make_config(2)
+    w2.Q *= -1.0
+    w2.dOut *= 0.5
+    pu.check_forward(w2, fb)
+    pu.check_backward(w2, fb, bb)
+
+
 def test_workspace_too_small_is_refused():
     w = wl.iid_workload("s", 82, [300], 1, 32, 8, wl.MODE_BF16_TC)
     Q, K, V, dO, offs = pu.to_device(w)
