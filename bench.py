@@ -258,6 +258,17 @@ def run_ours(args, w):
     kb.kmip_profile_enable(0)
     assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
 
+    # the same step replayed from a CUDA graph (launch overhead matters for the small configurations only)
+    graph_ms = None
+    try:
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg):
+            step()
+        cg.replay()
+        graph_ms = 1e3 * timed(cg.replay, args.steps) / args.steps
+    except Exception as exc:  # capture is an extra, never the measurement
+        graph_ms = f"capture failed: {exc}"
+
     e2e = e2e_setup()
     for _ in range(min(args.warmup, 2)):
         step_e2e()
@@ -321,6 +332,7 @@ def run_ours(args, w):
                 "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host.values())),
                 "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for n, t in host_out.items()
                                               if w.backward or n == "out"))},
+        "cuda_graph_replay_ms_per_step": graph_ms,
         "gpu_launches": (FWD_LAUNCHES + (BWD_LAUNCHES if w.backward else 0)) * args.steps,
         "clocks": clocks,
     }
