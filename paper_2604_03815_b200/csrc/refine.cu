@@ -145,9 +145,10 @@ cudaError_t launch_d(const FwdArgs& a, const T* keys) {
     refine_topk_kernel<T, D, E_, REGROUPED><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
         static_cast<const T*>(a.Q), keys, a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
         a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws))
-    // pending room CAP-k >= 96, so that the survivors of a row (rarely more than 2k) fit without
-    // intermediate compactions
-    if (a.k <= 32) KMIP_LAUNCH_REFINE(4);
+    // pending room CAP-k: the survivors of a row (rarely more than 2k) should fit without intermediate
+    // compactions, and the final sort costs log^2(CAP) compare-exchange stages
+    if (a.k <= 16) KMIP_LAUNCH_REFINE(2);
+    else if (a.k <= 32) KMIP_LAUNCH_REFINE(4);
     else KMIP_LAUNCH_REFINE(8);
 #undef KMIP_LAUNCH_REFINE
     return cudaGetLastError();
