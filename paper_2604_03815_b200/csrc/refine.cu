@@ -125,13 +125,14 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                     if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, jj[u]);
                     cnt += __popc(m);
                     if (cnt > room - 32) {
-                        tau = fmaxf(floor_tau, warp_compact_row<E>(row, k, cnt, lane));
+                        tau = fmaxf(floor_tau, E <= 4 ? warp_merge_row_chunks(row, k, cnt, lane) : warp_compact_row<E>(row, k, cnt, lane));
                         cnt = 0;
                     }
                 }
             }
         }
-        warp_compact_row<E>(row, k, cnt, lane);
+        // E <= 4 serves k <= 32: one kept key per lane, so the pending keys can be merged in 32-key chunks
+        if (E <= 4) warp_merge_row_chunks(row, k, cnt, lane); else warp_compact_row<E>(row, k, cnt, lane);
         warp_store_row(row, k, lane, topk_idx + (size_t)r * k, topk_score + (size_t)r * k);
     }
 }

@@ -119,6 +119,31 @@ __device__ __forceinline__ float warp_merge_row32(cand_t* row, int k, int cnt, i
     return kth ? cand_score(kth) : -CUDART_INF_F;
 }
 
+// Same result as warp_compact_row for k <= 32 and any cnt: the pending keys are taken 32 at a
+// time, each chunk is sorted on its own (one key per lane) and merged into the kept list as in
+// warp_merge_row32.  21 compare-exchange stages of one key per lane per chunk instead of
+// log^2(CAP) stages of CAP/32 keys per lane over the whole buffer.
+__device__ __forceinline__ float warp_merge_row_chunks(cand_t* row, int k, int cnt, int lane) {
+    __syncwarp();
+    cand_t m = (lane < k) ? row[lane] : 0ull;
+    for (int c0 = 0; c0 < cnt; c0 += 32) {
+        cand_t pend[1] = {(c0 + lane < cnt) ? row[k + c0 + lane] : 0ull};
+        warp_sort_desc<1>(pend, lane);
+        const cand_t rev = __shfl_sync(0xFFFFFFFFu, pend[0], 31 - lane);
+        m = cmax(m, rev);
+#pragma unroll
+        for (int j = 16; j > 0; j >>= 1) {
+            const cand_t o = __shfl_xor_sync(0xFFFFFFFFu, m, j);
+            m = ((lane & j) == 0) ? cmax(m, o) : cmin(m, o);
+        }
+    }
+    __syncwarp();
+    if (lane < k) row[lane] = m;
+    const cand_t kth = __shfl_sync(0xFFFFFFFFu, m, k - 1);
+    __syncwarp();
+    return kth ? cand_score(kth) : -CUDART_INF_F;
+}
+
 // Out-of-line entry points: compaction is rare, so one copy of its code is shared by all call
 // sites and stays out of the hot loop's instruction stream.
 template <int E>
