@@ -204,14 +204,36 @@ int kmip_oracle_forward_rows(const float *Q, const float *K, const float *V,
 }
 
 /*
+ * Attention dropout on the k softmax weights (the paper trains with it: 0.5 on the LRGB and
+ * City-Networks models, 0.0 on point clouds; App. G): each weight is kept with probability
+ * 1 - drop and divided by 1 - drop ("inverted" dropout), independently per (query, head, slot).
+ * The draw for slot t of query i, head h is a counter-based uniform: the splitmix64 finaliser
+ * of seed + (pair + 1) * 0x9E3779B97F4A7C15 with pair = (i*H + h)*k + t, top 24 bits / 2^24;
+ * the weight is kept when the uniform is >= drop.  Returns the factor the weight is multiplied by.
+ */
+static double dropout_factor(double drop, uint64_t seed, int64_t i, int32_t H, int32_t h, int32_t k, int t)
+{
+    if (drop <= 0.0)
+        return 1.0;
+    const uint64_t pair = ((uint64_t)i * (uint64_t)H + (uint64_t)h) * (uint64_t)k + (uint64_t)t;
+    uint64_t z = seed + (pair + 1u) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z = z ^ (z >> 31);
+    const double u = (double)(z >> 40) / 16777216.0;
+    return u >= drop ? 1.0 / (1.0 - drop) : 0.0;
+}
+
+/*
  * Lines 4-6 of Algorithm 1 for an index set supplied by the caller (any order, -1 = empty
- * slot); the scores of the listed keys are recomputed in fp64.
+ * slot); the scores of the listed keys are recomputed in fp64.  With drop > 0 the softmax
+ * weights go through dropout_factor (slot = position in idx) before the weighted sum.
  *   idx [n_rows, H, k], out [n_rows, H, d], score_out [n_rows, H, k] (optional).
  */
-int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V,
-                                  int64_t N, int32_t H, int32_t d, int32_t k,
-                                  const int64_t *rows, int64_t n_rows, const int32_t *idx,
-                                  double *out, double *score_out)
+int kmip_oracle_forward_given_idx_dropout(const float *Q, const float *K, const float *V,
+                                          int64_t N, int32_t H, int32_t d, int32_t k,
+                                          const int64_t *rows, int64_t n_rows, const int32_t *idx,
+                                          double drop, uint64_t seed, double *out, double *score_out)
 {
     if (!Q || !K || !V || !idx || !out || N < 0 || H < 1 || d < 1 || k < 1)
         return KMIP_ORACLE_BAD_ARG;
@@ -227,7 +249,8 @@ int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V
         double *s = (double *)malloc(sizeof(double) * (size_t)k);
         double *p = (double *)malloc(sizeof(double) * (size_t)k);
         int64_t *jj = (int64_t *)malloc(sizeof(int64_t) * (size_t)k);
-        if (!s || !p || !jj || i < 0 || i >= N) {
+        int *slot = (int *)malloc(sizeof(int) * (size_t)k);
+        if (!s || !p || !jj || !slot || i < 0 || i >= N) {
             failed = 1;
         } else {
             for (int32_t h = 0; h < H; ++h) {
@@ -244,6 +267,7 @@ int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V
                         continue;
                     }
                     jj[n] = ii[t];
+                    slot[n] = t;
                     s[n] = inner(q, K + jj[n] * HD + (int64_t)h * d, d);
                     if (score_out)
                         score_out[(r * H + h) * (int64_t)k + t] = s[n];
@@ -256,8 +280,9 @@ int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V
                     softmax_scaled(s, n, scale, p);
                     for (int t = 0; t < n; ++t) {
                         const float *v = V + jj[t] * HD + (int64_t)h * d;
+                        const double w = p[t] * dropout_factor(drop, seed, i, H, h, k, slot[t]);
                         for (int c = 0; c < d; ++c)
-                            o[c] += p[t] * (double)v[c];
+                            o[c] += w * (double)v[c];
                     }
                 }
             }
@@ -265,8 +290,17 @@ int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V
         free(s);
         free(p);
         free(jj);
+        free(slot);
     }
     return failed ? KMIP_ORACLE_BAD_ARG : KMIP_ORACLE_OK;
+}
+
+int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V,
+                                  int64_t N, int32_t H, int32_t d, int32_t k,
+                                  const int64_t *rows, int64_t n_rows, const int32_t *idx,
+                                  double *out, double *score_out)
+{
+    return kmip_oracle_forward_given_idx_dropout(Q, K, V, N, H, d, k, rows, n_rows, idx, 0.0, 0, out, score_out);
 }
 
 /*
@@ -276,10 +310,13 @@ int kmip_oracle_forward_given_idx(const float *Q, const float *K, const float *V
  *   dQ_i += dS_t k_{j_t}          dK_{j_t} += dS_t q_i      dV_{j_t} += p_t g_i
  * idx [N, H, k] (-1 = empty slot).  dQ, dK, dV [N, H, d] fp64, overwritten.
  * Heads touch disjoint columns, so the loop over heads is the parallel one.
+ * With dropout (factor f_t of dropout_factor, a constant of the backward pass) the output is
+ * o_i = sum_t f_t p_t v_{j_t}, so dP_t = f_t (g_i . v_{j_t}) and dV_{j_t} += f_t p_t g_i;
+ * D, dS, dQ and dK keep their form.
  */
-int kmip_oracle_backward(const float *Q, const float *K, const float *V, const float *dOut,
-                         const int32_t *idx, int64_t N, int32_t H, int32_t d, int32_t k,
-                         double *dQ, double *dK, double *dV)
+int kmip_oracle_backward_dropout(const float *Q, const float *K, const float *V, const float *dOut,
+                                 const int32_t *idx, int64_t N, int32_t H, int32_t d, int32_t k,
+                                 double drop, uint64_t seed, double *dQ, double *dK, double *dV)
 {
     if (!Q || !K || !V || !dOut || !idx || !dQ || !dK || !dV || N < 0 || H < 1 || d < 1 || k < 1)
         return KMIP_ORACLE_BAD_ARG;
@@ -296,7 +333,8 @@ int kmip_oracle_backward(const float *Q, const float *K, const float *V, const f
         double *p = (double *)malloc(sizeof(double) * (size_t)k);
         double *dP = (double *)malloc(sizeof(double) * (size_t)k);
         int64_t *jj = (int64_t *)malloc(sizeof(int64_t) * (size_t)k);
-        if (!s || !p || !dP || !jj) {
+        double *f = (double *)malloc(sizeof(double) * (size_t)k);
+        if (!s || !p || !dP || !jj || !f) {
             failed = 1;
         } else {
             for (int64_t i = 0; i < N; ++i) {
@@ -312,6 +350,7 @@ int kmip_oracle_backward(const float *Q, const float *K, const float *V, const f
                         continue;
                     }
                     jj[n] = ii[t];
+                    f[n] = dropout_factor(drop, seed, i, H, h, k, t);
                     s[n] = inner(q, K + jj[n] * HD + (int64_t)h * d, d);
                     ++n;
                 }
@@ -320,7 +359,7 @@ int kmip_oracle_backward(const float *Q, const float *K, const float *V, const f
                 softmax_scaled(s, n, scale, p);
                 double D = 0.0;
                 for (int t = 0; t < n; ++t) {
-                    dP[t] = inner(g, V + jj[t] * HD + (int64_t)h * d, d);
+                    dP[t] = f[t] * inner(g, V + jj[t] * HD + (int64_t)h * d, d);
                     D += p[t] * dP[t];
                 }
                 for (int t = 0; t < n; ++t) {
@@ -332,7 +371,7 @@ int kmip_oracle_backward(const float *Q, const float *K, const float *V, const f
                     for (int c = 0; c < d; ++c) {
                         dq[c] += dS * (double)kr[c];
                         dk[c] += dS * (double)q[c];
-                        dv[c] += p[t] * (double)g[c];
+                        dv[c] += f[t] * p[t] * (double)g[c];
                     }
                 }
             }
@@ -341,6 +380,14 @@ int kmip_oracle_backward(const float *Q, const float *K, const float *V, const f
         free(p);
         free(dP);
         free(jj);
+        free(f);
     }
     return failed ? KMIP_ORACLE_BAD_ARG : KMIP_ORACLE_OK;
+}
+
+int kmip_oracle_backward(const float *Q, const float *K, const float *V, const float *dOut,
+                         const int32_t *idx, int64_t N, int32_t H, int32_t d, int32_t k,
+                         double *dQ, double *dK, double *dV)
+{
+    return kmip_oracle_backward_dropout(Q, K, V, dOut, idx, N, H, d, k, 0.0, 0, dQ, dK, dV);
 }

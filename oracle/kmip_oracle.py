@@ -43,6 +43,11 @@ def _load():
         lib.kmip_oracle_forward_given_idx.argtypes = [P, P, P, i64, i32, i32, i32, P, i64, P, P, P]
         lib.kmip_oracle_backward.restype = ctypes.c_int
         lib.kmip_oracle_backward.argtypes = [P, P, P, P, P, i64, i32, i32, i32, P, P, P]
+        f64, u64 = ctypes.c_double, ctypes.c_uint64
+        lib.kmip_oracle_forward_given_idx_dropout.restype = ctypes.c_int
+        lib.kmip_oracle_forward_given_idx_dropout.argtypes = [P, P, P, i64, i32, i32, i32, P, i64, P, f64, u64, P, P]
+        lib.kmip_oracle_backward_dropout.restype = ctypes.c_int
+        lib.kmip_oracle_backward_dropout.argtypes = [P, P, P, P, P, i64, i32, i32, i32, f64, u64, P, P, P]
         _lib = lib
     return _lib
 
@@ -81,8 +86,9 @@ def forward(Q, K, V, graph_offsets, k, rows=None):
     return {"out": out, "idx": idx, "score": score, "gap": gap}
 
 
-def forward_given_idx(Q, K, V, idx, rows=None):
-    """Softmax-weighted sum over a caller-supplied index set; returns (out, score)."""
+def forward_given_idx(Q, K, V, idx, rows=None, drop=0.0, seed=0):
+    """Softmax-weighted sum over a caller-supplied index set (with attention dropout on the
+    weights when drop > 0); returns (out, score)."""
     Q, K, V = _f32(Q), _f32(K), _f32(V)
     N, H, d = Q.shape
     idx = np.ascontiguousarray(idx, dtype=np.int32)
@@ -92,15 +98,15 @@ def forward_given_idx(Q, K, V, idx, rows=None):
     k = idx.shape[2]
     out = np.zeros((n, H, d), dtype=np.float64)
     score = np.zeros((n, H, k), dtype=np.float64)
-    rc = _load().kmip_oracle_forward_given_idx(_ptr(Q), _ptr(K), _ptr(V), N, H, d, k,
-                                               _ptr(rws), n, _ptr(idx), _ptr(out), _ptr(score))
+    rc = _load().kmip_oracle_forward_given_idx_dropout(_ptr(Q), _ptr(K), _ptr(V), N, H, d, k, _ptr(rws), n, _ptr(idx),
+                                                       ctypes.c_double(drop), ctypes.c_uint64(seed), _ptr(out), _ptr(score))
     if rc != 0:
         raise ValueError(f"kmip_oracle_forward_given_idx failed with status {rc}")
     return out, score
 
 
-def backward(Q, K, V, dOut, idx):
-    """Sparse backward with the selection held constant; returns (dQ, dK, dV) in fp64."""
+def backward(Q, K, V, dOut, idx, drop=0.0, seed=0):
+    """Sparse backward with the selection (and the dropout draws) held constant; returns (dQ, dK, dV) in fp64."""
     Q, K, V, dOut = _f32(Q), _f32(K), _f32(V), _f32(dOut)
     N, H, d = Q.shape
     idx = np.ascontiguousarray(idx, dtype=np.int32)
@@ -109,8 +115,8 @@ def backward(Q, K, V, dOut, idx):
     dQ = np.empty((N, H, d), dtype=np.float64)
     dK = np.empty((N, H, d), dtype=np.float64)
     dV = np.empty((N, H, d), dtype=np.float64)
-    rc = _load().kmip_oracle_backward(_ptr(Q), _ptr(K), _ptr(V), _ptr(dOut), _ptr(idx), N, H, d, k,
-                                      _ptr(dQ), _ptr(dK), _ptr(dV))
+    rc = _load().kmip_oracle_backward_dropout(_ptr(Q), _ptr(K), _ptr(V), _ptr(dOut), _ptr(idx), N, H, d, k,
+                                              ctypes.c_double(drop), ctypes.c_uint64(seed), _ptr(dQ), _ptr(dK), _ptr(dV))
     if rc != 0:
         raise ValueError(f"kmip_oracle_backward failed with status {rc}")
     return dQ, dK, dV

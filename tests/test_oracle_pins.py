@@ -326,6 +326,87 @@ def test_backward_identities():
     assert np.all(dK[~hit] == 0) and np.all(dV[~hit] == 0)
 
 
+# ----------------------------------------------------------------------------- attention dropout
+def test_dropout_draws_follow_the_published_generator():
+    """Slot t of query 0, head 0 draws the (t+1)-th SplitMix64 output for the seed (fixture: the
+    generator's published vector for state 0).  Three equal scores give weights 1/3 in key order,
+    so with drop = 0.5 the output is the sum of (1/3) / 0.5 * v_t over the slots whose top 24 bits
+    are at least half of 2^24."""
+    import json, os
+    fx = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "splitmix64_vectors.json")))
+    u = [int(x, 16) >> 40 for x in fx["outputs_hex"][:3]]
+    keep = [x >= (1 << 23) for x in u]
+    assert keep == [True, False, False]
+    N, H, d, k = 3, 1, 4, 3
+    Q = np.zeros((N, H, d), dtype=np.float32)
+    K = np.ones((N, H, d), dtype=np.float32)
+    V = np.arange(N * d, dtype=np.float32).reshape(N, H, d) + 1.0
+    idx = np.tile(np.arange(3, dtype=np.int32), (N, H, 1))
+    out, _ = oracle.forward_given_idx(Q, K, V, idx, drop=0.5, seed=fx["initial_state"])
+    want = sum((1.0 / 3.0) / 0.5 * V[t, 0].astype(np.float64) for t in range(3) if keep[t])
+    np.testing.assert_allclose(out[0, 0], want, rtol=1e-14)
+
+
+def test_dropout_zero_is_the_plain_path_and_keep_rate_matches():
+    sizes, H, d, k = [300], 2, 8, 1
+    Q, K, V, g = _rand(31, sizes[0], H, d)
+    f = oracle.forward(Q, K, V, _offs(*sizes), k)
+    plain, _ = oracle.forward_given_idx(Q, K, V, f["idx"])
+    same, _ = oracle.forward_given_idx(Q, K, V, f["idx"], drop=0.0, seed=123)
+    assert np.array_equal(plain, same)
+    # k = 1: the single weight is 1, so a row is either v / (1 - drop) or exactly zero
+    drop = 0.3
+    out, _ = oracle.forward_given_idx(Q, K, V, f["idx"], drop=drop, seed=9)
+    zero = np.all(out == 0.0, axis=-1)
+    np.testing.assert_allclose(out[~zero], plain[~zero] / (1.0 - drop), rtol=1e-14)
+    n = zero.size
+    assert abs(zero.mean() - drop) < 5.0 * np.sqrt(drop * (1 - drop) / n)      # binomial, 5 sigma
+    again, _ = oracle.forward_given_idx(Q, K, V, f["idx"], drop=drop, seed=9)
+    other, _ = oracle.forward_given_idx(Q, K, V, f["idx"], drop=drop, seed=10)
+    assert np.array_equal(out, again) and not np.array_equal(out, other)
+
+
+def test_dropout_is_unbiased():
+    """Constant V = 1: the output is the sum of the dropped-out weights, with expectation 1 and
+    variance sum_t p_t^2 * drop / (1 - drop) <= drop / (1 - drop); averaged over S seeds."""
+    sizes, H, d, k = [60], 2, 4, 6
+    Q, K, _, _ = _rand(32, sizes[0], H, d)
+    V = np.ones((sizes[0], H, d), dtype=np.float32)
+    f = oracle.forward(Q, K, V, _offs(*sizes), k)
+    drop, S = 0.5, 400
+    acc = np.zeros((sizes[0], H, d))
+    for s in range(S):
+        acc += oracle.forward_given_idx(Q, K, V, f["idx"], drop=drop, seed=1000 + s)[0]
+    assert np.all(np.abs(acc / S - 1.0) < 6.0 * np.sqrt(drop / (1 - drop) / S))
+
+
+def test_dropout_backward_matches_finite_differences():
+    """L = sum(out * g) with the selection and the draws held fixed is a smooth function of Q, K, V:
+    central differences in fp64 pin the backward formulas with dropout (dP scaled, dV scaled)."""
+    sizes, H, d, k = [9, 6], 2, 3, 4
+    N = sum(sizes)
+    Q, K, V, g = _rand(33, N, H, d)
+    f = oracle.forward(Q, K, V, _offs(*sizes), k)
+    idx, drop, seed = f["idx"], 0.4, 77
+    dQ, dK, dV = oracle.backward(Q, K, V, g, idx, drop=drop, seed=seed)
+
+    def loss(q, kk, v):
+        return float((oracle.forward_given_idx(q, kk, v, idx, drop=drop, seed=seed)[0] * g.astype(np.float64)).sum())
+
+    rng = np.random.default_rng(5)
+    eps = 2.0 ** -8          # exactly representable steps keep the float32 inputs exact
+    for name, grad in (("Q", dQ), ("K", dK), ("V", dV)):
+        for _ in range(12):
+            i, h, c = rng.integers(N), rng.integers(H), rng.integers(d)
+            args = {"Q": Q.copy(), "K": K.copy(), "V": V.copy()}
+            args[name][i, h, c] += eps
+            up = loss(args["Q"], args["K"], args["V"])
+            args[name][i, h, c] -= 2 * eps
+            dn = loss(args["Q"], args["K"], args["V"])
+            num = (up - dn) / (2 * eps)
+            assert abs(num - grad[i, h, c]) <= 2e-4 * max(1.0, abs(num)), (name, i, h, c, num, grad[i, h, c])
+
+
 # ----------------------------------------------------------------------------- argument checks
 def test_bad_arguments_are_rejected():
     Q, K, V, _ = _rand(26, 8, 1, 4)
