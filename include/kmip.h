@@ -112,6 +112,35 @@ int kmip_attn_backward(const void *Q, const void *K, const void *V,
                        void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Training variants with attention dropout on the k softmax weights (the paper trains its LRGB and
+ * City-Networks models with attention dropout 0.5 and its point-cloud models with 0; App. G).
+ * Each weight p_t of Algorithm 1 line 5 is kept with probability 1 - drop_p and divided by
+ * 1 - drop_p, independently per (query, head, slot):
+ *   out[i,h,:] = sum_t f_t p_t V[topk_idx_t, h, :],   f_t = 1/(1 - drop_p) or 0.
+ * The draws are counter based, so the backward call regenerates them from the same (drop_p, seed)
+ * and nothing is stored: slot t of query i, head h uses the ((i*H + h)*k + t + 1)-th output of
+ * SplitMix64 started at `seed`; its top 24 bits / 2^24 is the uniform, kept when >= drop_p.
+ * topk_idx and topk_score are not affected.  In the backward pass f is a constant:
+ *   dP_t = f_t (g_i . v_{j_t}),  dV gets f_t p_t g_i,  D, dS, dQ, dK as in kmip_attn_backward.
+ * drop_p must be in [0, 1) (else KMIP_ERR_INVALID_ARG); drop_p = 0 is exactly kmip_attn_forward /
+ * kmip_attn_backward.  All other arguments, layouts, ownership and errors are theirs.
+ */
+int kmip_attn_forward_dropout(const void *Q, const void *K, const void *V,
+                              const int32_t *graph_offsets, int32_t G, int64_t N,
+                              int32_t H, int32_t d, int32_t k, int mode,
+                              float drop_p, uint64_t seed,
+                              void *out, int32_t *topk_idx, float *topk_score,
+                              void *workspace, size_t workspace_bytes, void *stream);
+int kmip_attn_backward_dropout(const void *Q, const void *K, const void *V,
+                               const int32_t *graph_offsets, int32_t G, int64_t N,
+                               int32_t H, int32_t d, int32_t k, int mode,
+                               float drop_p, uint64_t seed,
+                               const void *out, const void *d_out,
+                               const int32_t *topk_idx, const float *topk_score,
+                               void *dQ, void *dK, void *dV,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Size in bytes of the scratch array that is built into the library for
  * kmip_attn_forward_static_scratch (8 MiB; each GPU that loads the library holds it until the
  * process exits).

@@ -54,6 +54,12 @@ def lib() -> ctypes.CDLL:
         L.kmip_attn_backward.restype = ctypes.c_int
         L.kmip_attn_backward.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, P, P, P, P,
                                          P, P, P, P, sz, P]
+        f32, u64 = ctypes.c_float, ctypes.c_uint64
+        L.kmip_attn_forward_dropout.restype = ctypes.c_int
+        L.kmip_attn_forward_dropout.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, f32, u64, P, P, P, P, sz, P]
+        L.kmip_attn_backward_dropout.restype = ctypes.c_int
+        L.kmip_attn_backward_dropout.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, f32, u64, P, P, P, P,
+                                                 P, P, P, P, sz, P]
         L.kmip_last_status.restype = ctypes.c_int
         L.kmip_last_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_int)]
         L.kmip_attn_forward_static_scratch.restype = ctypes.c_int
@@ -101,6 +107,30 @@ def kmip_attn_forward(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score
                                        _ptr(out), _ptr(topk_idx), _ptr(topk_score), _ptr(workspace),
                                        0 if workspace is None else workspace.numel() * workspace.element_size(),
                                        _stream(stream)))
+
+
+def kmip_attn_forward_dropout(Q, K, V, graph_offsets, k, mode, drop_p, seed, out, topk_idx, topk_score, workspace,
+                              stream=None) -> int:
+    """Forward pass with attention dropout on the k softmax weights (counter-based draws from `seed`)."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(lib().kmip_attn_forward_dropout(_ptr(Q), _ptr(K), _ptr(V), _ptr(graph_offsets), G, N, H, d, k, mode,
+                                               float(drop_p), int(seed), _ptr(out), _ptr(topk_idx), _ptr(topk_score),
+                                               _ptr(workspace),
+                                               0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                               _stream(stream)))
+
+
+def kmip_attn_backward_dropout(Q, K, V, graph_offsets, k, mode, drop_p, seed, out, d_out, topk_idx, topk_score,
+                               dQ, dK, dV, workspace, stream=None) -> int:
+    """Backward pass of kmip_attn_forward_dropout with the same (drop_p, seed)."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(lib().kmip_attn_backward_dropout(_ptr(Q), _ptr(K), _ptr(V), _ptr(graph_offsets), G, N, H, d, k, mode,
+                                                float(drop_p), int(seed), _ptr(out), _ptr(d_out), _ptr(topk_idx),
+                                                _ptr(topk_score), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(workspace),
+                                                0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                                _stream(stream)))
 
 
 def kmip_attn_forward_static_scratch(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score,

@@ -65,8 +65,17 @@ int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_
 int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
                       int64_t N, int32_t H, int32_t d, int32_t k, int mode, void* out, int32_t* topk_idx,
                       float* topk_score, void* workspace, size_t workspace_bytes, void* stream) {
+    return kmip_attn_forward_dropout(Q, K, V, graph_offsets, G, N, H, d, k, mode, 0.0f, 0ull, out, topk_idx, topk_score,
+                                     workspace, workspace_bytes, stream);
+}
+
+int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
+                              int64_t N, int32_t H, int32_t d, int32_t k, int mode, float drop_p, uint64_t seed,
+                              void* out, int32_t* topk_idx, float* topk_score, void* workspace,
+                              size_t workspace_bytes, void* stream) {
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
+    if (!(drop_p >= 0.0f && drop_p < 1.0f)) return KMIP_ERR_INVALID_ARG;
     if (N == 0) return KMIP_OK;
     if (graph_offsets != nullptr && G < 1) return KMIP_ERR_INVALID_ARG;
     if (!Q || !K || !V || !out || !topk_idx || !topk_score || !workspace) return KMIP_ERR_INVALID_ARG;
@@ -79,6 +88,8 @@ int kmip_attn_forward(const void* Q, const void* K, const void* V, const int32_t
 
     FwdArgs a{Q, K, V, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, out, topk_idx, topk_score,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    a.drop_p = drop_p;
+    a.seed = seed;
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
@@ -105,9 +116,18 @@ int kmip_attn_backward(const void* Q, const void* K, const void* V, const int32_
                        int64_t N, int32_t H, int32_t d, int32_t k, int mode, const void* out, const void* d_out,
                        const int32_t* topk_idx, const float* topk_score, void* dQ, void* dK, void* dV,
                        void* workspace, size_t workspace_bytes, void* stream) {
+    return kmip_attn_backward_dropout(Q, K, V, graph_offsets, G, N, H, d, k, mode, 0.0f, 0ull, out, d_out, topk_idx,
+                                      topk_score, dQ, dK, dV, workspace, workspace_bytes, stream);
+}
+
+int kmip_attn_backward_dropout(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
+                               int64_t N, int32_t H, int32_t d, int32_t k, int mode, float drop_p, uint64_t seed,
+                               const void* out, const void* d_out, const int32_t* topk_idx, const float* topk_score,
+                               void* dQ, void* dK, void* dV, void* workspace, size_t workspace_bytes, void* stream) {
     (void)graph_offsets; (void)G; (void)out;
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
+    if (!(drop_p >= 0.0f && drop_p < 1.0f)) return KMIP_ERR_INVALID_ARG;
     if (N == 0) return KMIP_OK;
     if (!Q || !K || !V || !d_out || !topk_idx || !topk_score || !dQ || !dK || !dV || !workspace)
         return KMIP_ERR_INVALID_ARG;
@@ -118,6 +138,8 @@ int kmip_attn_backward(const void* Q, const void* K, const void* V, const int32_
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
     BwdArgs a{Q, K, V, d_out, N, H, d, k, mode, topk_idx, topk_score, dQ, dK, dV,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    a.drop_p = drop_p;
+    a.seed = seed;
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_bwd < g_prof.max_calls) ? g_prof.bwd[g_prof.n_bwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);

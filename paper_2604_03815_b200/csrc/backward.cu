@@ -24,7 +24,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 bwd_rows_kernel(const T* __restrict__ K, const T* __restrict__ V, const T* __restrict__ dOut,
                 const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_score,
-                int N, int H, int k, float scale,
+                int N, int H, int k, float scale, float drop_p, unsigned long long seed,
                 float* __restrict__ ws_p, float* __restrict__ ws_ds, T* __restrict__ dQ) {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;
@@ -56,6 +56,16 @@ bwd_rows_kernel(const T* __restrict__ K, const T* __restrict__ V, const T* __res
                 }
             }
         }
+        // with dropout the output was sum_t f_t p_t v_t (f constant here): dP_t = f_t (g . v_t), and the
+        // weight that reaches dV is f_t p_t
+        float f[kMaxEntriesPerLane];
+#pragma unroll
+        for (int e = 0; e < kMaxEntriesPerLane; ++e) f[e] = 1.0f;
+        if (drop_p > 0.0f) {
+            dropout_factors(r, k, lane, drop_p, seed, f);
+#pragma unroll
+            for (int e = 0; e < kMaxEntriesPerLane; ++e) dP[e] *= f[e];
+        }
         float dsum = 0.0f;
 #pragma unroll
         for (int e = 0; e < kMaxEntriesPerLane; ++e) dsum = fmaf(p[e], dP[e], dsum);
@@ -66,7 +76,7 @@ bwd_rows_kernel(const T* __restrict__ K, const T* __restrict__ V, const T* __res
             dS[e] = scale * p[e] * (dP[e] - dsum);
             const int t = e * 32 + lane;
             if (t < k) {
-                ws_p[(size_t)r * k + t] = p[e];
+                ws_p[(size_t)r * k + t] = f[e] * p[e];
                 ws_ds[(size_t)r * k + t] = dS[e];
             }
         }
@@ -377,7 +387,8 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
 
     const int row_blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
     bwd_rows_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
-        K, V, dOut, a.topk_idx, a.topk_score, (int)a.N, a.H, a.k, scale, ws_p, ws_ds, static_cast<T*>(a.dQ));
+        K, V, dOut, a.topk_idx, a.topk_score, (int)a.N, a.H, a.k, scale, a.drop_p, a.seed, ws_p, ws_ds,
+        static_cast<T*>(a.dQ));
     if (ev) cudaEventRecord(ev[0], a.stream);
 
     const int pair_blocks = (int)((n_pairs + 255) / 256);

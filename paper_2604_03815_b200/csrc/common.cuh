@@ -144,6 +144,8 @@ struct FwdArgs {
     float* topk_score;
     unsigned char* ws;
     cudaStream_t stream;
+    float drop_p = 0.0f;             // attention dropout on the k weights (0 = none)
+    unsigned long long seed = 0ull;  // of its counter-based draws
 };
 
 struct BwdArgs {
@@ -156,6 +158,8 @@ struct BwdArgs {
     void *dQ, *dK, *dV;
     unsigned char* ws;
     cudaStream_t stream;
+    float drop_p = 0.0f;
+    unsigned long long seed = 0ull;
 };
 
 // plan.cu: validates the offsets and writes the work items of the tensor-core kernel

@@ -15,7 +15,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 softmax_gather_kernel(const T* __restrict__ V, const int32_t* __restrict__ topk_idx,
                       const float* __restrict__ topk_score, int N, int H, int k, float scale,
-                      T* __restrict__ out, const StatusBlock* __restrict__ sb) {
+                      float drop_p, unsigned long long seed, T* __restrict__ out,
+                      const StatusBlock* __restrict__ sb) {
     if (sb->status != KMIP_OK) return;  // an earlier stage failed: topk_idx was not written
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;
@@ -27,6 +28,12 @@ softmax_gather_kernel(const T* __restrict__ V, const int32_t* __restrict__ topk_
         int j[kMaxEntriesPerLane];
         float p[kMaxEntriesPerLane];
         load_row_softmax(topk_idx + (size_t)r * k, topk_score + (size_t)r * k, k, N, scale, lane, j, p);
+        if (drop_p > 0.0f) {  // training only: the weights go through dropout before the weighted sum
+            float f[kMaxEntriesPerLane];
+            dropout_factors(r, k, lane, drop_p, seed, f);
+#pragma unroll
+            for (int e = 0; e < kMaxEntriesPerLane; ++e) p[e] *= f[e];
+        }
         float acc[VEC];
         gather_weighted_sum<T, D>(V, H, h, k, lane, j, p, acc);
         if (lane < LPR) Elem<T>::store_vec(out + (size_t)r * D + lane * VEC, acc);
@@ -39,7 +46,7 @@ cudaError_t launch_d(const FwdArgs& a) {
     const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
     softmax_gather_kernel<T, D><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         static_cast<const T*>(a.V), a.topk_idx, a.topk_score, (int)a.N, a.H, a.k,
-        1.0f / sqrtf((float)a.d), static_cast<T*>(a.out), reinterpret_cast<const StatusBlock*>(a.ws));
+        1.0f / sqrtf((float)a.d), a.drop_p, a.seed, static_cast<T*>(a.out), reinterpret_cast<const StatusBlock*>(a.ws));
     return cudaGetLastError();
 }
 

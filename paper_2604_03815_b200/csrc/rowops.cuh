@@ -54,6 +54,24 @@ __device__ __forceinline__ void load_row_softmax(const int32_t* idx_row, const f
     for (int e = 0; e < kMaxEntriesPerLane; ++e) p[e] *= inv;
 }
 
+// Attention dropout on the k weights of row r (= query * H + head): factor 1/(1-drop) when the slot's
+// counter-based uniform is >= drop, else 0.  The draw of slot t is the (r*k + t + 1)-th SplitMix64
+// output for `seed`, top 24 bits / 2^24.  f[e] belongs to entry t = e*32 + lane.
+__device__ __forceinline__ void dropout_factors(long long r, int k, int lane, float drop, unsigned long long seed,
+                                                float (&f)[kMaxEntriesPerLane]) {
+    const float keep_scale = 1.0f / (1.0f - drop);
+#pragma unroll
+    for (int e = 0; e < kMaxEntriesPerLane; ++e) {
+        const unsigned long long pair = (unsigned long long)r * (unsigned long long)k + (unsigned long long)(e * 32 + lane);
+        unsigned long long z = seed + (pair + 1ull) * 0x9E3779B97F4A7C15ull;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        z = z ^ (z >> 31);
+        const float u = (float)(unsigned)(z >> 40) * (1.0f / 16777216.0f);  // 24 bits: exact in fp32
+        f[e] = (u >= drop) ? keep_scale : 0.0f;
+    }
+}
+
 // acc (per lane: VEC columns of the part this lane owns) = sum_t w_t * X[j_t, h, part*VEC ..].
 // LPR = D/VEC lanes share one gathered row (one 16-byte load each), 32/LPR rows per round.
 // After the call lanes 0..LPR-1 hold the full sums for their part.

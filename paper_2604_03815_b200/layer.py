@@ -19,11 +19,18 @@ class KMIPAttentionFunction(torch.autograd.Function):
     """out = kMIP-Attn(Q, K, V) over CSR-batched graphs; Q, K, V: [N, H, d] contiguous."""
 
     @staticmethod
-    def forward(ctx, Q, K, V, graph_offsets, k, mode):
+    def forward(ctx, Q, K, V, graph_offsets, k, mode, drop_p=0.0, seed=0):
         Q, K, V = Q.contiguous(), K.contiguous(), V.contiguous()
-        fb = kb.forward(Q, K, V, graph_offsets, k, mode, check=False)
+        N, H, d = Q.shape
+        G = 1 if graph_offsets is None else int(graph_offsets.numel()) - 1
+        fb = kb.ForwardBuffers(N, G, H, d, k, mode, Q.device)
+        rc = kb.kmip_attn_forward_dropout(Q, K, V, graph_offsets, k, mode, drop_p, seed, fb.out, fb.topk_idx,
+                                          fb.topk_score, fb.workspace)
+        if rc != kb.KMIP_OK:
+            raise kb.KmipError(rc, "kmip_attn_forward_dropout")
         ctx.save_for_backward(Q, K, V, fb.out, fb.topk_idx, fb.topk_score)
         ctx.graph_offsets, ctx.k, ctx.mode, ctx.fwd_workspace = graph_offsets, k, mode, fb.workspace
+        ctx.drop_p, ctx.seed = drop_p, seed
         ctx.mark_non_differentiable(fb.topk_idx)
         return fb.out, fb.topk_idx
 
@@ -33,14 +40,17 @@ class KMIPAttentionFunction(torch.autograd.Function):
         st = kb.kmip_last_status(ctx.fwd_workspace)  # device-side problems of the forward surface here at the latest
         if st != kb.KMIP_OK:
             raise kb.KmipError(st, "kmip_attn_forward (device)")
-        fwd = _Saved(out, topk_idx, topk_score)
-        bb = kb.backward(Q, K, V, ctx.graph_offsets, ctx.k, ctx.mode, fwd, d_out.contiguous(), check=True)
-        return bb.dQ, bb.dK, bb.dV, None, None, None
-
-
-class _Saved:
-    def __init__(self, out, topk_idx, topk_score):
-        self.out, self.topk_idx, self.topk_score = out, topk_idx, topk_score
+        N, H, d = Q.shape
+        G = 1 if ctx.graph_offsets is None else int(ctx.graph_offsets.numel()) - 1
+        bb = kb.BackwardBuffers(N, G, H, d, ctx.k, ctx.mode, Q.device)
+        rc = kb.kmip_attn_backward_dropout(Q, K, V, ctx.graph_offsets, ctx.k, ctx.mode, ctx.drop_p, ctx.seed, out,
+                                           d_out.contiguous(), topk_idx, topk_score, bb.dQ, bb.dK, bb.dV, bb.workspace)
+        if rc != kb.KMIP_OK:
+            raise kb.KmipError(rc, "kmip_attn_backward_dropout")
+        st = kb.kmip_last_status(bb.workspace)
+        if st != kb.KMIP_OK:
+            raise kb.KmipError(st, "kmip_attn_backward_dropout (device)")
+        return bb.dQ, bb.dK, bb.dV, None, None, None, None, None
 
 
 class KMIPSelfAttention(torch.nn.Module):
@@ -48,13 +58,19 @@ class KMIPSelfAttention(torch.nn.Module):
     O^h = kMIP-Attn(Q^h, K^h, V^h) restricted to each graph, y = sum_h O^h W_O^h (Eq. 2).
 
     d_head must be 16, 32, 64 or 128 and k <= 128.  dtype bfloat16 selects the tensor-core mode,
-    float32 the fp32 mode."""
+    float32 the fp32 mode.  attn_dropout is the dropout rate on the k attention weights, active in
+    training mode only (the paper's graph models use 0.5); every forward call draws a fresh seed
+    from torch's CPU generator, so torch.manual_seed makes a run repeatable."""
 
-    def __init__(self, d_model, num_heads, d_head, k, dtype=torch.bfloat16, device="cuda", bias=False):
+    def __init__(self, d_model, num_heads, d_head, k, dtype=torch.bfloat16, device="cuda", bias=False,
+                 attn_dropout=0.0):
         super().__init__()
         if dtype not in (torch.bfloat16, torch.float32):
             raise ValueError("dtype must be torch.bfloat16 or torch.float32")
         self.d_model, self.H, self.d, self.k = d_model, num_heads, d_head, k
+        if not 0.0 <= attn_dropout < 1.0:
+            raise ValueError("attn_dropout must be in [0, 1)")
+        self.attn_dropout = float(attn_dropout)
         self.mode = kb.KMIP_BF16_TC if dtype == torch.bfloat16 else kb.KMIP_FP32_EXACT
         inner = num_heads * d_head
         self.w_q = torch.nn.Linear(d_model, inner, bias=bias, device=device, dtype=dtype)
@@ -69,6 +85,8 @@ class KMIPSelfAttention(torch.nn.Module):
         q = self.w_q(x).view(N, self.H, self.d)
         k = self.w_k(x).view(N, self.H, self.d)
         v = self.w_v(x).view(N, self.H, self.d)
-        o, idx = KMIPAttentionFunction.apply(q, k, v, graph_offsets, self.k, self.mode)
+        drop = self.attn_dropout if self.training else 0.0
+        seed = int(torch.randint(0, 2 ** 62, (1,)).item()) if drop > 0.0 else 0
+        o, idx = KMIPAttentionFunction.apply(q, k, v, graph_offsets, self.k, self.mode, drop, seed)
         y = self.w_o(o.reshape(N, self.H * self.d))
         return (y, idx) if return_indices else y

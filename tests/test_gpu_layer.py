@@ -81,3 +81,24 @@ def test_layer_forward_and_gradients(dtype, d_head, k):
     close(x.grad, x64.grad, "d/dx")
     for p, w64, name in zip((layer.w_q.weight, layer.w_k.weight, layer.w_v.weight, layer.w_o.weight), ws, "QKVO"):
         close(p.grad, w64.grad, f"d/dW_{name}")
+
+
+def test_layer_attention_dropout_only_in_training():
+    from paper_2604_03815_b200.layer import KMIPSelfAttention
+
+    torch.manual_seed(7)
+    layer = KMIPSelfAttention(32, 2, 16, 8, attn_dropout=0.5)
+    x = torch.randn(300, 32, device="cuda").to(torch.bfloat16)
+    layer.eval()
+    a, b = layer(x), layer(x)
+    assert torch.equal(a, b)
+    layer.train()
+    torch.manual_seed(11)
+    c = layer(x)
+    torch.manual_seed(11)
+    d = layer(x)
+    e = layer(x)
+    assert torch.equal(c, d) and not torch.equal(c, e) and not torch.equal(c, a)
+    xg = x.clone().requires_grad_(True)
+    layer(xg).float().square().sum().backward()
+    assert torch.isfinite(xg.grad.float()).all() and float(xg.grad.float().abs().max()) > 0
