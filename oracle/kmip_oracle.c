@@ -204,6 +204,66 @@ int kmip_oracle_forward_rows(const float *Q, const float *K, const float *V,
 }
 
 /*
+ * Diagnostic of the paper's App. H ("cumulative attention weight"): how much of the FULL softmax
+ * over all keys of the query's graph falls on the k keys with the largest scores,
+ *   mass[i,h] = sum_{t<k} softmax_j(q_i.k_j / sqrt(d))_(t)     (1 when the graph has <= k nodes).
+ * Plain definition: every score of the row, a stable log-sum-exp over all of them, and the sum of
+ * the k largest probabilities.  mass [n_rows, H] fp64, indexed by position in `rows`.
+ */
+static int cmp_desc(const void *a, const void *b)
+{
+    const double x = *(const double *)a, y = *(const double *)b;
+    return (x < y) - (x > y);
+}
+
+int kmip_oracle_topk_mass(const float *Q, const float *K, const int32_t *graph_offsets, int32_t G, int64_t N,
+                          int32_t H, int32_t d, int32_t k, const int64_t *rows, int64_t n_rows, double *mass)
+{
+    if (!Q || !K || !mass || N < 0 || H < 1 || d < 1 || k < 1)
+        return KMIP_ORACLE_BAD_ARG;
+    if (!offsets_ok(graph_offsets, G, N))
+        return KMIP_ORACLE_BAD_ARG;
+    if (rows == NULL)
+        n_rows = N;
+    const double scale = 1.0 / sqrt((double)d);
+    const int64_t HD = (int64_t)H * d;
+    int failed = 0;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const int64_t i = rows ? rows[r] : r;
+        int64_t lo, hi;
+        if (i < 0 || i >= N || !graph_range(graph_offsets, G, N, i, &lo, &hi)) {
+            failed = 1;
+            continue;
+        }
+        const int64_t n = hi - lo;
+        double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+        if (!s) {
+            failed = 1;
+            continue;
+        }
+        for (int32_t h = 0; h < H; ++h) {
+            const float *q = Q + i * HD + (int64_t)h * d;
+            double m = -INFINITY, z = 0.0, top = 0.0;
+            for (int64_t j = lo; j < hi; ++j) {
+                s[j - lo] = scale * inner(q, K + j * HD + (int64_t)h * d, d);
+                if (s[j - lo] > m)
+                    m = s[j - lo];
+            }
+            for (int64_t j = 0; j < n; ++j)
+                z += exp(s[j] - m);
+            qsort(s, (size_t)n, sizeof(double), cmp_desc);
+            for (int64_t t = 0; t < n && t < k; ++t)
+                top += exp(s[t] - m);
+            mass[r * H + h] = n > 0 ? top / z : 0.0;
+        }
+        free(s);
+    }
+    return failed ? KMIP_ORACLE_BAD_ARG : KMIP_ORACLE_OK;
+}
+
+/*
  * Attention dropout on the k softmax weights (the paper trains with it: 0.5 on the LRGB and
  * City-Networks models, 0.0 on point clouds; App. G): each weight is kept with probability
  * 1 - drop and divided by 1 - drop ("inverted" dropout), independently per (query, head, slot).

@@ -44,6 +44,8 @@ def _load():
         lib.kmip_oracle_backward.restype = ctypes.c_int
         lib.kmip_oracle_backward.argtypes = [P, P, P, P, P, i64, i32, i32, i32, P, P, P]
         f64, u64 = ctypes.c_double, ctypes.c_uint64
+        lib.kmip_oracle_topk_mass.restype = ctypes.c_int
+        lib.kmip_oracle_topk_mass.argtypes = [P, P, P, i32, i64, i32, i32, i32, P, i64, P]
         lib.kmip_oracle_forward_given_idx_dropout.restype = ctypes.c_int
         lib.kmip_oracle_forward_given_idx_dropout.argtypes = [P, P, P, i64, i32, i32, i32, P, i64, P, f64, u64, P, P]
         lib.kmip_oracle_backward_dropout.restype = ctypes.c_int
@@ -120,3 +122,19 @@ def backward(Q, K, V, dOut, idx, drop=0.0, seed=0):
     if rc != 0:
         raise ValueError(f"kmip_oracle_backward failed with status {rc}")
     return dQ, dK, dV
+
+
+def topk_mass(Q, K, graph_offsets, k, rows=None):
+    """Share of the full softmax (over all keys of the query's graph) that falls on the k largest
+    scores; [n_rows, H] fp64."""
+    Q, K = _f32(Q), _f32(K)
+    N, H, d = Q.shape
+    offs = None if graph_offsets is None else np.ascontiguousarray(graph_offsets, dtype=np.int32)
+    G = 1 if offs is None else len(offs) - 1
+    rws = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = N if rws is None else len(rws)
+    mass = np.zeros((n, H), dtype=np.float64)
+    rc = _load().kmip_oracle_topk_mass(_ptr(Q), _ptr(K), _ptr(offs), G, N, H, d, k, _ptr(rws), n, _ptr(mass))
+    if rc != 0:
+        raise ValueError(f"kmip_oracle_topk_mass failed with status {rc}")
+    return mass

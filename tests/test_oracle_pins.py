@@ -407,6 +407,31 @@ def test_dropout_backward_matches_finite_differences():
             assert abs(num - grad[i, h, c]) <= 2e-4 * max(1.0, abs(num)), (name, i, h, c, num, grad[i, h, c])
 
 
+# ----------------------------------------------------------------------------- top-k mass diagnostic
+def test_topk_mass_against_library_softmax_and_special_cases():
+    from scipy.special import softmax
+    sizes, H, d, k = [37, 5, 60], 2, 8, 7
+    N = sum(sizes)
+    Q, K, _, _ = _rand(41, N, H, d)
+    Q *= 3.0                                       # peaked rows as well as flat ones
+    offs = _offs(*sizes)
+    mass = oracle.topk_mass(Q, K, offs, k)
+    for g in range(len(sizes)):
+        lo, hi = offs[g], offs[g + 1]
+        for h in range(H):
+            S = Q[lo:hi, h].astype(np.float64) @ K[lo:hi, h].astype(np.float64).T / np.sqrt(d)
+            P = np.sort(softmax(S, axis=1), axis=1)[:, ::-1]
+            np.testing.assert_allclose(mass[lo:hi, h], P[:, :k].sum(axis=1), rtol=1e-12)
+    np.testing.assert_allclose(mass[37:42], 1.0, rtol=1e-14)   # a graph with fewer nodes than k keeps everything
+    # identical keys: every probability is 1/n, so the k largest hold k/n
+    K2 = np.repeat(K[:1], N, axis=0)
+    m2 = oracle.topk_mass(Q, K2, offs, k)
+    np.testing.assert_allclose(m2[:37], k / 37.0, rtol=1e-12)
+    np.testing.assert_allclose(m2[42:], k / 60.0, rtol=1e-12)
+    # monotone in k and equal to the kept weights of the forward pass relative to the full softmax
+    assert np.all(oracle.topk_mass(Q, K, offs, k + 3) >= mass - 1e-15)
+
+
 # ----------------------------------------------------------------------------- argument checks
 def test_bad_arguments_are_rejected():
     Q, K, V, _ = _rand(26, 8, 1, 4)
