@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.kmip_attn_backward_dropout.restype = ctypes.c_int
         L.kmip_attn_backward_dropout.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, f32, u64, P, P, P, P,
                                                  P, P, P, P, sz, P]
+        L.kmip_attn_topk_mass.restype = ctypes.c_int
+        L.kmip_attn_topk_mass.argtypes = [P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, P, P, P, sz, P]
         L.kmip_last_status.restype = ctypes.c_int
         L.kmip_last_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_int)]
         L.kmip_attn_forward_static_scratch.restype = ctypes.c_int
@@ -131,6 +133,16 @@ def kmip_attn_backward_dropout(Q, K, V, graph_offsets, k, mode, drop_p, seed, ou
                                                 _ptr(topk_score), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(workspace),
                                                 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                                 _stream(stream)))
+
+
+def kmip_attn_topk_mass(Q, K, graph_offsets, k, mode, topk_score, mass, workspace, stream=None) -> int:
+    """Share of the full softmax held by the kept scores, [N, H] float32 (diagnostic; one more pass over all scores)."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(lib().kmip_attn_topk_mass(_ptr(Q), _ptr(K), _ptr(graph_offsets), G, N, H, d, k, mode, _ptr(topk_score),
+                                         _ptr(mass), _ptr(workspace),
+                                         0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                         _stream(stream)))
 
 
 def kmip_attn_forward_static_scratch(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score,

@@ -147,6 +147,28 @@ int kmip_attn_backward_dropout(const void* Q, const void* K, const void* V, cons
     return KMIP_OK;
 }
 
+int kmip_attn_topk_mass(const void* Q, const void* K, const int32_t* graph_offsets, int32_t G, int64_t N, int32_t H,
+                        int32_t d, int32_t k, int mode, const float* topk_score, float* mass, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    const int rc = check_shape(N, H, d, k, mode);
+    if (rc != KMIP_OK) return rc;
+    if (d > 64) return KMIP_ERR_UNSUPPORTED;
+    if (N == 0) return KMIP_OK;
+    if (graph_offsets != nullptr && G < 1) return KMIP_ERR_INVALID_ARG;
+    if (!Q || !K || !topk_score || !mass || !workspace) return KMIP_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(topk_score) || !aligned16(workspace) ||
+        (reinterpret_cast<uintptr_t>(mass) & 3u) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
+        return KMIP_ERR_INVALID_ARG;
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, false);
+    if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
+    FwdArgs a{Q, K, nullptr, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, nullptr, nullptr,
+              const_cast<float*>(topk_score), static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_plan(a, w, 128) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_topk_mass(a, w, mass) != cudaSuccess) return KMIP_ERR_CUDA;
+    return KMIP_OK;
+}
+
 int kmip_last_status(const void* workspace, void* stream, int* device_status) {
     if (!workspace || !device_status) return KMIP_ERR_INVALID_ARG;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;

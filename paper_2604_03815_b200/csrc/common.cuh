@@ -180,6 +180,8 @@ cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float*
 // refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k
 cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_refine_topk_fp32(const FwdArgs& a);
+// topk_mass.cu: share of the full softmax held by the kept scores; needs 128-row work items in the workspace
+cudaError_t launch_topk_mass(const FwdArgs& a, const FwdWorkspace& w, float* mass);
 // tiled CUDA-core sweep of fp32 mode (score_select_fp32.cu): 128-row work items, then launch_refine_topk_fp32
 bool score_select_fp32_tiled_supported(int32_t d, int32_t k);
 cudaError_t launch_score_select_fp32_tiled(const FwdArgs& a, const FwdWorkspace& w);
