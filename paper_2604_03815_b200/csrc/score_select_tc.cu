@@ -374,20 +374,21 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 for (int j = 0; ok && j < ntiles; ++j, ++kt) {
                     const int s = kt % S;
                     const uint64_t stage_off = (uint64_t)((s * Sh::TILE_BYTES) >> 4);  // start-address field counts 16-byte units
-                    bool have_keys = false;
+                    // Both issuers wait for EVERY key tile, also one whose pairs all belong to the other
+                    // issuer (one query tile per CTA): a parity wait is sound only on a barrier whose
+                    // every phase the waiter observes, and with an odd number of stages an issuer that
+                    // skipped its partner's tiles would meet a stage only every second time it is filled.
+                    long long c0 = (dbg & 8) ? clock64() : 0;
+                    if (!(ok = wait_or_abort<0>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
+                    if (dbg & 8) w_kfull += clock64() - c0;
 #pragma unroll
                     for (int qt = 0; qt < NQT; ++qt) {
                         const int seq = kt * NQT + qt;
                         if ((seq & 1) != mine) continue;
                         const int b = seq & (NBUF - 1);
-                        long long c0 = (dbg & 8) ? clock64() : 0;
-                        if (!have_keys) {
-                            if (!(ok = wait_or_abort<0>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
-                            have_keys = true;
-                        }
                         long long c1 = (dbg & 8) ? clock64() : 0;
                         if (!(ok = wait_or_abort<0>(bars.t_empty(b), ((seq >> 2) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
-                        if (dbg & 8) { w_kfull += c1 - c0; w_tempty += clock64() - c1; }
+                        if (dbg & 8) w_tempty += clock64() - c1;
                         ptx::tc_fence_after();
                         if (qt < nq) {
                             const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
