@@ -78,3 +78,31 @@ def test_large_runs_are_bit_identical(cfg, kw):
             ref = cur
         else:
             assert all(torch.equal(a, b) for a, b in zip(ref, cur))
+
+
+def test_random_small_shapes_against_the_oracle():
+    """Random small batches through every path (tensor-core sweep, both fp32 sweeps, the per-row kernel
+    with bf16 storage), forward and backward, each held to the full parity bar against the oracle."""
+    from tests import parity_util as pu
+
+    rng = np.random.default_rng(5)
+    for case in range(80):
+        H = int(rng.integers(1, 4))
+        d = int(rng.choice([16, 32, 64, 128]))
+        k = int(rng.choice([1, 2, 5, 8, 16, 31, 32, 33, 48, 64, 100, 128]))
+        if d == 128 and k > 64:
+            k = int(rng.choice([1, 7, 64, 100]))
+        sizes = rng.integers(0, int(rng.choice([10, 140, 600, 1500])), size=int(rng.integers(1, 12))).tolist()
+        if sum(sizes) == 0:
+            sizes[0] = 3
+        mode = wl.MODE_BF16_TC if rng.random() < 0.7 else wl.MODE_FP32_EXACT
+        path = int(rng.integers(0, 3)) if mode == wl.MODE_FP32_EXACT else 0
+        w = wl.iid_workload("s", 700000 + case, sizes, H, d, k, mode, input_scale=float(rng.choice([0.2, 1.0])) / np.sqrt(d))
+        kb.lib().kmip_debug_fp32_path(path)
+        try:
+            dev = pu.to_device(w)
+            fb = pu.run_forward(w, dev)
+            pu.check_forward(w, fb)
+            pu.check_backward(w, fb, pu.run_backward(w, fb, dev))
+        finally:
+            kb.lib().kmip_debug_fp32_path(0)
