@@ -61,7 +61,7 @@ typedef enum {
  * Scratch size in bytes that kmip_attn_forward (pass = 0) or kmip_attn_backward (pass = 1)
  * needs for this problem size.  Linear in N*H*(k + d): the N x N score matrix of Algorithm 1
  * line 2 is never stored (Sec. 3.1, App. F).  Forward: one bf16 copy of K regrouped by head
- * (tensor-core mode only) plus the work list; backward: 12 bytes per selected pair plus
+ * (tensor-core mode only) plus the work list; backward: 24 bytes per selected pair plus
  * 12 bytes per (node, head).  Host only, no CUDA call.
  */
 int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k,

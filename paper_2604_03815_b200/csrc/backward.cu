@@ -205,28 +205,32 @@ scan_write_kernel(int* __restrict__ counts, long long n, const int* __restrict__
     }
 }
 
+// A hit record of the key-major lists: everything the segment reduction needs about one selected
+// pair in one 16-byte load - the query row, its softmax weight p (times the dropout factor) and its
+// score gradient dS - instead of a pair id that would cost two more scattered 4-byte reads per hit.
 __global__ void fill_kernel(const int32_t* __restrict__ topk_idx, long long n_pairs, int N, int H, int k,
-                            const int* __restrict__ seg_off, int* __restrict__ cursor, int* __restrict__ pairs) {
+                            const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
+                            const int* __restrict__ seg_off, int* __restrict__ cursor, int4* __restrict__ hits) {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_pairs) return;
     const int j = __ldg(topk_idx + e);
     if (j < 0 || j >= N) return;
-    const int h = (int)((e / k) % H);
+    const long long r = e / k;  // query * H + head
+    const int h = (int)(r % H);
     const size_t key = (size_t)j * H + h;
-    pairs[seg_off[key] + atomicAdd(cursor + key, 1)] = (int)e;
+    hits[seg_off[key] + atomicAdd(cursor + key, 1)] =
+        make_int4((int)(r / H), __float_as_int(__ldg(ws_p + e)), __float_as_int(__ldg(ws_ds + e)), 0);
 }
 
 // -------------------------------------------------------------------------------------- segments
-// Accumulate one hit (pair id e) into the lane's part of dV and dK.
+// Accumulate one hit into the lane's part of dV and dK.
 template <typename T, int D>
-__device__ __forceinline__ void accumulate_hit(int e, int HK, int h, int H, int part,
+__device__ __forceinline__ void accumulate_hit(int4 rec, int h, int H, int part,
                                                const T* __restrict__ Q, const T* __restrict__ dOut,
-                                               const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
                                                float (&accV)[Elem<T>::kVec], float (&accK)[Elem<T>::kVec]) {
     constexpr int VEC = Elem<T>::kVec;
-    const int i = e / HK;
-    const float pw = __ldg(ws_p + e), dsw = __ldg(ws_ds + e);
-    const size_t off = ((size_t)i * H + h) * D + part * VEC;
+    const float pw = __int_as_float(rec.y), dsw = __int_as_float(rec.z);
+    const size_t off = ((size_t)rec.x * H + h) * D + part * VEC;
     float gv[VEC], qv[VEC];
     Elem<T>::load_vec(dOut + off, gv);
     Elem<T>::load_vec(Q + off, qv);
@@ -238,52 +242,47 @@ __device__ __forceinline__ void accumulate_hit(int e, int HK, int h, int H, int 
 }
 
 // Accumulates the hits first, first+stride, ... (< len) of one list; four hits are in flight at a time
-// so that the dependent loads (pair id -> weights and rows) of different hits overlap.
+// so that the dependent loads (record -> rows) of different hits overlap.
 template <typename T, int D>
-__device__ __forceinline__ void accumulate_list(const int* __restrict__ list, int first, int stride, int len, int HK,
+__device__ __forceinline__ void accumulate_list(const int4* __restrict__ list, int first, int stride, int len,
                                                 int h, int H, int part, const T* __restrict__ Q,
-                                                const T* __restrict__ dOut, const float* __restrict__ ws_p,
-                                                const float* __restrict__ ws_ds, float (&accV)[Elem<T>::kVec],
+                                                const T* __restrict__ dOut, float (&accV)[Elem<T>::kVec],
                                                 float (&accK)[Elem<T>::kVec]) {
     constexpr int VEC = Elem<T>::kVec;
     int t = first;
     for (; t + 3 * stride < len; t += 4 * stride) {
-        int e[4];
-        float pw[4], dsw[4], gv[4][VEC], qv[4][VEC];
+        int4 rec[4];
+        float gv[4][VEC], qv[4][VEC];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) e[u] = __ldg(list + t + u * stride);
+        for (int u = 0; u < 4; ++u) rec[u] = __ldg(list + t + u * stride);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const size_t off = ((size_t)(e[u] / HK) * H + h) * D + part * VEC;
-            pw[u] = __ldg(ws_p + e[u]);
-            dsw[u] = __ldg(ws_ds + e[u]);
+            const size_t off = ((size_t)rec[u].x * H + h) * D + part * VEC;
             Elem<T>::load_vec(dOut + off, gv[u]);
             Elem<T>::load_vec(Q + off, qv[u]);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
+            const float pw = __int_as_float(rec[u].y), dsw = __int_as_float(rec[u].z);
 #pragma unroll
             for (int c = 0; c < VEC; ++c) {
-                accV[c] = fmaf(pw[u], gv[u][c], accV[c]);
-                accK[c] = fmaf(dsw[u], qv[u][c], accK[c]);
+                accV[c] = fmaf(pw, gv[u][c], accV[c]);
+                accK[c] = fmaf(dsw, qv[u][c], accK[c]);
             }
         }
     }
-    for (; t < len; t += stride)
-        accumulate_hit<T, D>(__ldg(list + t), HK, h, H, part, Q, dOut, ws_p, ws_ds, accV, accK);
+    for (; t < len; t += stride) accumulate_hit<T, D>(__ldg(list + t), h, H, part, Q, dOut, accV, accK);
 }
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 bwd_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
-                    const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
-                    const int* __restrict__ seg_off, const int* __restrict__ pairs,
+                    const int* __restrict__ seg_off, const int4* __restrict__ hits,
                     long long n_segs, int H, int k, T* __restrict__ dK, T* __restrict__ dV) {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;
     constexpr int EPW = 32 / LPR;
     const int lane = threadIdx.x & 31, part = lane % LPR, sub = lane / LPR;
-    const int HK = H * k;
     for (long long x = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); x < n_segs;
          x += (long long)gridDim.x * kWarpsPerBlock) {
         const int start = __ldg(seg_off + x), len = __ldg(seg_off + x + 1) - start;
@@ -292,7 +291,7 @@ bwd_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
         float accV[VEC], accK[VEC];
 #pragma unroll
         for (int c = 0; c < VEC; ++c) { accV[c] = 0.0f; accK[c] = 0.0f; }
-        accumulate_list<T, D>(pairs + start, sub, EPW, len, HK, h, H, part, Q, dOut, ws_p, ws_ds, accV, accK);
+        accumulate_list<T, D>(hits + start, sub, EPW, len, h, H, part, Q, dOut, accV, accK);
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
@@ -311,8 +310,7 @@ bwd_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
 template <typename T, int D>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 bwd_long_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
-                         const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
-                         const int* __restrict__ seg_off, const int* __restrict__ pairs,
+                         const int* __restrict__ seg_off, const int4* __restrict__ hits,
                          const int* __restrict__ long_list, const StatusBlock* __restrict__ sb,
                          int H, int k, T* __restrict__ dK, T* __restrict__ dV) {
     constexpr int VEC = Elem<T>::kVec;
@@ -320,7 +318,6 @@ bwd_long_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
     constexpr int EPW = 32 / LPR;
     __shared__ float s_part[kWarpsPerBlock][2][D];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, part = lane % LPR, sub = lane / LPR;
-    const int HK = H * k;
     const int n_long = sb->n_long;
     for (int li = blockIdx.x; li < n_long; li += gridDim.x) {
         const int x = __ldg(long_list + li);
@@ -329,8 +326,7 @@ bwd_long_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
         float accV[VEC], accK[VEC];
 #pragma unroll
         for (int c = 0; c < VEC; ++c) { accV[c] = 0.0f; accK[c] = 0.0f; }
-        accumulate_list<T, D>(pairs + start, wid * EPW + sub, kWarpsPerBlock * EPW, len, HK, h, H, part, Q, dOut, ws_p,
-                              ws_ds, accV, accK);
+        accumulate_list<T, D>(hits + start, wid * EPW + sub, kWarpsPerBlock * EPW, len, h, H, part, Q, dOut, accV, accK);
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
@@ -375,7 +371,7 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     float* ws_ds = reinterpret_cast<float*>(a.ws + w.ds_off);
     int* seg_off = reinterpret_cast<int*>(a.ws + w.seg_off);
     int* cursor = reinterpret_cast<int*>(a.ws + w.cursor_off);
-    int* pairs = reinterpret_cast<int*>(a.ws + w.pairs_off);
+    int4* hits = reinterpret_cast<int4*>(a.ws + w.pairs_off);
     int* block_sums = reinterpret_cast<int*>(a.ws + w.blocksum_off);
     int* long_list = reinterpret_cast<int*>(a.ws + w.long_off);
     const T *Q = static_cast<const T*>(a.Q), *K = static_cast<const T*>(a.K), *V = static_cast<const T*>(a.V);
@@ -396,13 +392,14 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     scan_block_sums_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums);
     scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(block_sums, w.scan_blocks);
     scan_write_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums, seg_off, long_list, sb);
-    fill_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, seg_off, cursor, pairs);
+    fill_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, ws_p, ws_ds, seg_off, cursor,
+                                                  hits);
     if (ev) cudaEventRecord(ev[1], a.stream);
 
     bwd_segments_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
-        Q, dOut, ws_p, ws_ds, seg_off, pairs, n_rows, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
+        Q, dOut, seg_off, hits, n_rows, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
     bwd_long_segments_kernel<T, D><<<148 * 8, kWarpsPerBlock * 32, 0, a.stream>>>(
-        Q, dOut, ws_p, ws_ds, seg_off, pairs, long_list, sb, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
+        Q, dOut, seg_off, hits, long_list, sb, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
     if (ev) cudaEventRecord(ev[2], a.stream);
     return cudaGetLastError();
 }

@@ -58,7 +58,7 @@ struct BwdWorkspace {
     size_t ds_off;        // float [N*H*k]   score gradients
     size_t seg_off;       // int   [N*H+1]   start of each (key, head) hit list
     size_t cursor_off;    // int   [N*H]     hit counts, then fill cursors
-    size_t pairs_off;     // int   [N*H*k]   hit lists: flat pair ids (i*H+h)*k+t
+    size_t pairs_off;     // int4  [N*H*k]   hit lists: records {query row, p, dS, 0}
     size_t blocksum_off;  // int   [scan blocks]
     size_t long_off;      // int   [N*H]     ids of long segments
     size_t total;
@@ -76,7 +76,7 @@ inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
     w.ds_off = o;       o = align_up(o + 4 * pairs);
     w.seg_off = o;      o = align_up(o + 4 * (rows + 1));
     w.cursor_off = o;   o = align_up(o + 4 * (rows + 1));
-    w.pairs_off = o;    o = align_up(o + 4 * pairs);
+    w.pairs_off = o;    o = align_up(o + 16 * pairs);
     w.blocksum_off = o; o = align_up(o + 4 * (size_t)(w.scan_blocks + 1));
     w.long_off = o;     o = align_up(o + 4 * rows);
     w.total = o;

@@ -278,5 +278,5 @@ def test_workspace_too_small_is_refused():
 def test_workspace_is_linear_in_n():
     a = kb.kmip_attn_workspace_bytes(100_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
     b = kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
-    assert b < 10.5 * a and b < 1_000_000 * 4 * (3 * 16 + 4) * 4 + (1 << 20)
+    assert b < 10.5 * a and b < 1_000_000 * 4 * (6 * 16 + 4) * 4 + (1 << 20)   # 24 bytes per selected pair + per-row arrays
     assert kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_FORWARD) < 1_000_000 * 4 * 32 * 2 + (1 << 20)
