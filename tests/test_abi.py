@@ -44,7 +44,7 @@ def test_workspace_bytes_host_only(kb):
     assert 500_000 * 4 * 32 * 2 < f < 500_000 * 4 * 32 * 2 + (1 << 20)   # K regrouped by head + work items
     assert 256 < kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_FP32_EXACT, kb.PASS_FORWARD) < (1 << 20)
     pairs = 500_000 * 4 * 32
-    assert 12 * pairs < b < 14 * pairs          # p, dS, pair list: 12 bytes per selected pair + O(N*H)
+    assert 24 * pairs < b < 26 * pairs          # p, dS, 16-byte hit records: 24 bytes per selected pair + O(N*H)
     for bad in [dict(d=24), dict(k=129), dict(mode=7)]:
         args = dict(N=1000, G=1, H=2, d=32, k=8, mode=kb.KMIP_BF16_TC)
         args.update(bad)
