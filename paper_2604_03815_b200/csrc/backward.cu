@@ -319,10 +319,14 @@ bwd_long_segments_kernel(const T* __restrict__ Q, const T* __restrict__ dOut,
     __shared__ float s_part[kWarpsPerBlock][2][D];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, part = lane % LPR, sub = lane / LPR;
     const int n_long = sb->n_long;
+    // Head by head: the dO and Q rows of one head (N * d elements each) fit the L2 cache, those of
+    // all heads together do not, and a query row is gathered k times across the lists of a head.
+    for (int hp = 0; hp < H; ++hp)
     for (int li = blockIdx.x; li < n_long; li += gridDim.x) {
         const int x = __ldg(long_list + li);
-        const int start = __ldg(seg_off + x), len = __ldg(seg_off + x + 1) - start;
         const int h = x % H;
+        if (h != hp) continue;  // block-uniform
+        const int start = __ldg(seg_off + x), len = __ldg(seg_off + x + 1) - start;
         float accV[VEC], accK[VEC];
 #pragma unroll
         for (int c = 0; c < VEC; ++c) { accV[c] = 0.0f; accK[c] = 0.0f; }
