@@ -310,12 +310,17 @@ def run_ours(args, w):
     esz = 2 if w.mode == wl.MODE_BF16_TC else 4
     bwd_bytes = pairs * (4 * w.d * esz + 28) + 7 * w.N * w.H * w.d * esz
     fwd_tail_bytes = w.N * w.H * (w.k * (8 + w.d * esz) + w.d * esz)
+    arr_mb = w.N * w.H * w.d * esz / 1e6
+    l2_note = (f"Q, K, V, dOut and the outputs ({arr_mb:.0f} MB each) exceed the 126 MB L2; no flush between steps"
+               if arr_mb > 126 else
+               f"Q, K, V, dOut and the outputs are {arr_mb:.1f} MB each and fit the 126 MB L2; no flush between steps, "
+               "so this is a cache-warm figure (the headline workload is config 4)")
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.mode == wl.MODE_BF16_TC else "f32", "data": "synthetic",
         "config": {"workload": describe(w), "passes": "forward+backward" if w.backward else "forward",
-                   "l2": "Q, K, V, dOut and the outputs (>=128 MB each) exceed the 126 MB L2; no flush between steps",
+                   "l2": l2_note,
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": roofline,
         "stages_ms": {k_: round(v, 4) for k_, v in per_call.items()},
