@@ -60,7 +60,8 @@ typedef enum {
 /*
  * Scratch size in bytes that kmip_attn_forward (pass = 0) or kmip_attn_backward (pass = 1)
  * needs for this problem size.  Linear in N*H*(k + d): the N x N score matrix of Algorithm 1
- * line 2 is never stored (Sec. 3.1, App. F).  Forward: one bf16 copy of K regrouped by head
+ * line 2 is never stored (Sec. 3.1, App. F).  Forward: one bf16 copy of K regrouped by head and, from
+ * 32768 nodes on, one of Q in the sweep's row order plus 6 bytes per node
  * (tensor-core mode only) plus the work list; backward: 24 bytes per selected pair plus
  * 12 bytes per (node, head).  Host only, no CUDA call.
  */
@@ -175,7 +176,8 @@ int kmip_attn_topk_mass(const void *Q, const void *K,
  *   - there is no workspace argument: the scratch is a fixed KMIP_STATIC_SCRATCH_BYTES array inside
  *     the library.  A problem whose kmip_attn_workspace_bytes(..., KMIP_PASS_FORWARD) exceeds it is
  *     refused with KMIP_ERR_TOO_LARGE before anything is enqueued.  In tensor-core mode the scratch
- *     is dominated by one bf16 copy of K, so the limit is about N*H*d <= 4.1 million elements
+ *     is dominated by one bf16 copy of K (and one of Q from 32768 nodes on), so the limit is about
+ *     N*H*d <= 4.1 million elements (2 million from 32768 nodes on)
  *     (e.g. 32 000 nodes at H = 4, d = 32); fp32 mode needs 16 bytes per 128 nodes and per graph.
  *   - device_status (DEVICE pointer, may be NULL): if given, the device status word of this call
  *     (KMIP_OK, KMIP_ERR_TIMEOUT or KMIP_ERR_BAD_OFFSETS) is copied there on `stream` after the

@@ -99,6 +99,7 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
     const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k) &&
                          (g_fp32_path == 0 ? (N / 128) * H >= 296 : g_fp32_path == 2);
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (w.reorder && launch_reorder_queries(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
     const cudaError_t sweep = tc ? launch_score_select_tc(a, w)
                               : tiled32 ? launch_score_select_fp32_tiled(a, w) : launch_score_select_exact(a);

@@ -39,9 +39,15 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a = kAlign) { return
 struct FwdWorkspace {
     size_t items_off;  // WorkItem[max_items]
     size_t kpack_off;  // bf16 [H, N, d]: K regrouped by head for the tensor-core sweep (0 bytes otherwise)
+    size_t qperm_off;  // bf16 [N, H, d]: Q in the sweep's row order (only when `reorder`)
+    size_t perm_off;   // int  [N]: original row of each sweep row
+    size_t code_off;   // u16  [N]: locality codes of the query rows
     size_t total;
     int max_items;
+    bool reorder;      // the sweep runs the rows of large graphs in locality order (reorder.cu)
 };
+
+constexpr int64_t kReorderMinNodes = 32768;  // below this the extra launches cost more than they can save
 
 // `tc`: the tensor-core sweep will run (bf16 mode and a supported (d, k))
 inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, bool tc) {
@@ -49,7 +55,11 @@ inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t 
     w.max_items = (int)(N / 128 + (G > 0 ? G : 1) + 1);
     w.items_off = kStatusBytes;
     w.kpack_off = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
-    w.total = align_up(w.kpack_off + (tc ? (size_t)N * H * d * 2 : 0));
+    w.reorder = tc && N >= kReorderMinNodes;
+    w.qperm_off = align_up(w.kpack_off + (tc ? (size_t)N * H * d * 2 : 0));
+    w.perm_off = align_up(w.qperm_off + (w.reorder ? (size_t)N * H * d * 2 : 0));
+    w.code_off = align_up(w.perm_off + (w.reorder ? (size_t)N * 4 : 0));
+    w.total = align_up(w.code_off + (w.reorder ? (size_t)N * 2 : 0));
     return w;
 }
 
@@ -166,6 +176,8 @@ struct BwdArgs {
 cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_item);
 // plan.cu: K [N, H, d] -> [H, N, d] so that a head's key tile is one contiguous block for TMA
 cudaError_t launch_pack_keys(const FwdArgs& a, const FwdWorkspace& w);
+// reorder.cu: locality codes, per-graph bucket sort, row-permuted copy of Q (after launch_plan)
+cudaError_t launch_reorder_queries(const FwdArgs& a, const FwdWorkspace& w);
 // score_select_exact.cu: CUDA-core scores + running top-k, any supported (d, k), fp32 or bf16 storage
 cudaError_t launch_score_select_exact(const FwdArgs& a);
 // score_select_tc.cu: tcgen05 scores + running top-k (bf16 storage); returns cudaErrorNotSupported

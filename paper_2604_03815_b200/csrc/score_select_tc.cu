@@ -248,7 +248,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
                        float* __restrict__ dump, int dump_ld /* = N */, int dbg_arg, long long* __restrict__ timing,
-                       long long wait_limit, int drop_first_tile) {
+                       long long wait_limit, int drop_first_tile, const int* __restrict__ perm) {
     const int dbg = kSweepDebug ? dbg_arg : 0;
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
@@ -556,7 +556,8 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 __syncwarp();
                 const int nloc = min(32, it.nrows - (qt * BM + quarter * 32));
                 for (int r = 0; r < nloc; ++r) {
-                    const size_t o = ((size_t)(it.row0 + qt * BM + quarter * 32 + r) * H + h) * k;
+                    const int srow = it.row0 + qt * BM + quarter * 32 + r;  // sweep order; the result goes to the row's own place
+                    const size_t o = ((size_t)(perm ? __ldg(perm + srow) : srow) * H + h) * k;
                     for (int t = lane; t < k; t += 32) {
                         const uint32_t c = wl[t * 32 + r];
                         topk_idx[o + t] = c ? (int)wl[Sp::LIST * 32 + t * 32 + r] : -1;
@@ -644,7 +645,7 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
                                   (size_t)Sp::NBARS * 8 + 16 + 64;
     static_assert(smem_bytes <= 232448, "shared memory budget of one CTA");
     CUtensorMap tmQ, tmK;
-    if (!make_tensor_map<D>(&tmQ, a.Q, a.N, (int64_t)a.H * D) ||
+    if (!make_tensor_map<D>(&tmQ, w.reorder ? static_cast<const void*>(a.ws + w.qperm_off) : a.Q, a.N, (int64_t)a.H * D) ||
         !make_tensor_map<D>(&tmK, a.ws + w.kpack_off, a.N * a.H, D))
         return cudaErrorInvalidValue;
     auto kern = score_select_tc_kernel<D, KG, NQT, S, DUMP>;
@@ -655,7 +656,7 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
         a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing, g_wait_limit_cycles,
-        g_drop_first_tile);
+        g_drop_first_tile, (w.reorder && !DUMP) ? reinterpret_cast<const int*>(a.ws + w.perm_off) : nullptr);
     return cudaGetLastError();
 }
 

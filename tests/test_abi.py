@@ -41,7 +41,10 @@ def test_version_and_status_strings(kb):
 def test_workspace_bytes_host_only(kb):
     f = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
     b = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
-    assert 500_000 * 4 * 32 * 2 < f < 500_000 * 4 * 32 * 2 + (1 << 20)   # K regrouped by head + work items
+    kq = 2 * 500_000 * 4 * 32 * 2                                           # bf16 copies of K (regrouped) and Q (sweep order)
+    assert kq < f < kq + 500_000 * 6 + (1 << 20)                           # + permutation, codes, work items
+    small = kb.kmip_attn_workspace_bytes(20_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
+    assert 20_000 * 4 * 32 * 2 < small < 20_000 * 4 * 32 * 2 + (1 << 20)    # small problems keep their row order: K copy only
     assert 256 < kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_FP32_EXACT, kb.PASS_FORWARD) < (1 << 20)
     pairs = 500_000 * 4 * 32
     assert 24 * pairs < b < 26 * pairs          # p, dS, 16-byte hit records: 24 bytes per selected pair + O(N*H)
