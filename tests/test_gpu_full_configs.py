@@ -45,3 +45,27 @@ def test_config4_500k_point_cloud():
 def test_config5_hub_batch():
     st = _full(5, 256)
     assert st["identical_rows"] > 0.95
+
+
+def test_mixed_batch_with_reordered_and_untouched_graphs():
+    """From 32768 nodes on, the sweep runs the rows of graphs with at least 8192 nodes in locality
+    order and leaves smaller graphs alone; every row's result must still land at the row's own
+    place.  Clustered queries (so that the order really changes), all rows checked for structure,
+    a stratified sample against the oracle, the backward pass in full."""
+    sizes = [9000, 300, 20000, 10, 8192, 4000, 0, 8191]
+    base = wl.make_config(4, N=sum(sizes), H=2, d=32, k=16)
+    offs = np.zeros(len(sizes) + 1, dtype=np.int64)
+    np.cumsum(sizes, out=offs[1:])
+    w = wl.Workload(name="mixed", mode=base.mode, H=base.H, d=base.d, k=base.k, graph_offsets=offs.astype(np.int32),
+                    Q=base.Q, K=base.K, V=base.V, dOut=base.dOut, backward=True, meta={})
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    rows = wl.sample_rows(w, 400)
+    pu.check_forward(w, fb, rows)
+    idx = fb.topk_idx.cpu().numpy()
+    g = np.searchsorted(offs, np.arange(w.N), side="right") - 1
+    keff = np.minimum(w.k, offs[g + 1] - offs[g])[:, None, None]
+    valid = np.arange(w.k)[None, None, :] < keff
+    assert np.all(((idx >= offs[g][:, None, None]) & (idx < offs[g + 1][:, None, None])) | ~valid)
+    assert np.all((idx == -1) | valid)
+    pu.check_backward(w, fb, pu.run_backward(w, fb, dev))
