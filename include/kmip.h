@@ -51,7 +51,16 @@ typedef enum {
        accumulation on the tcgen05 tensor cores; softmax, sums and gradients accumulate in fp32. */
     KMIP_BF16_TC = 0,
     /* All of them hold fp32.  Scores are fp32 fused multiply-adds in index order c = 0..d-1. */
-    KMIP_FP32_EXACT = 1
+    KMIP_FP32_EXACT = 1,
+    /* KMIP_BF16_TC with an exact pruning of the search (the quadratic search is the first limitation the
+       paper names, Sec. 6): in graphs of 8192 nodes or more the keys are swept in an order that puts heavy
+       and similar keys together, and a 128-key tile is skipped for a block of query rows when a bound on
+       every inner product of the pair (centroids and radii, or Cauchy-Schwarz with the largest key norm)
+       lies below all of the block's current k-th best scores.  Same results as KMIP_BF16_TC up to the
+       order in which equal scores are met; forward only differs, the backward pass is the same.
+       Needs about 16 more bytes per node, 4 per (node, head) and (d + 4) * 4 * H per 128 nodes of scratch.
+       Below 32768 nodes it is KMIP_BF16_TC. */
+    KMIP_BF16_TC_PRUNED = 2
 } kmip_mode_t;
 
 #define KMIP_PASS_FORWARD 0

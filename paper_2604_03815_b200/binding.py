@@ -21,6 +21,7 @@ KMIP_ERR_BAD_OFFSETS = 6
 KMIP_ERR_TOO_LARGE = 7
 KMIP_BF16_TC = 0
 KMIP_FP32_EXACT = 1
+KMIP_BF16_TC_PRUNED = 2
 PASS_FORWARD = 0
 PASS_BACKWARD = 1
 
@@ -209,7 +210,7 @@ def kmip_debug_tc_scores(Q, K, scores, workspace, stream=None) -> int:
 # Buffer helpers (allocation only)
 # ------------------------------------------------------------------------------------------------
 def storage_dtype(mode: int):
-    return torch.bfloat16 if mode == KMIP_BF16_TC else torch.float32
+    return torch.float32 if mode == KMIP_FP32_EXACT else torch.bfloat16
 
 
 class ForwardBuffers:

@@ -10,7 +10,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int check_shape(int64_t N, int32_t H, int32_t d, int32_t k, int mode) {
     if (N < 0 || N >= (int64_t)1 << 31 || H < 1 || k < 1 || d < 1) return KMIP_ERR_INVALID_ARG;
-    if (mode != KMIP_BF16_TC && mode != KMIP_FP32_EXACT) return KMIP_ERR_UNSUPPORTED;
+    if (mode != KMIP_BF16_TC && mode != KMIP_FP32_EXACT && mode != KMIP_BF16_TC_PRUNED) return KMIP_ERR_UNSUPPORTED;
     if (d != 16 && d != 32 && d != 64 && d != 128) return KMIP_ERR_UNSUPPORTED;
     if (k > 128) return KMIP_ERR_UNSUPPORTED;
     if ((__int128)N * H * k >= (__int128)1 << 31) return KMIP_ERR_INVALID_ARG;
@@ -56,7 +56,8 @@ int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
     if (pass == KMIP_PASS_FORWARD)
-        *bytes = plan_fwd_workspace(N, G, H, d, mode == KMIP_BF16_TC && score_select_tc_supported(d, k)).total;
+        *bytes = plan_fwd_workspace(N, G, H, d, mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k),
+                                    mode == KMIP_BF16_TC_PRUNED).total;
     else if (pass == KMIP_PASS_BACKWARD) *bytes = plan_bwd_workspace(N, H, k).total;
     else return KMIP_ERR_INVALID_ARG;
     return KMIP_OK;
@@ -82,8 +83,8 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || !aligned16(topk_idx) ||
         !aligned16(topk_score) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
         return KMIP_ERR_INVALID_ARG;
-    const bool tc = mode == KMIP_BF16_TC && score_select_tc_supported(d, k);
-    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, tc);
+    const bool tc = mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k);
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, tc, mode == KMIP_BF16_TC_PRUNED);
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
 
     FwdArgs a{Q, K, V, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, out, topk_idx, topk_score,
@@ -93,13 +94,14 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
-    if (tc && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (tc && !w.prune && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     // the tiled fp32 sweep runs one block per 128 query rows and head: worth it once that fills the GPU
     // about twice, below that the one-warp-per-row kernel has more parallelism
     const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k) &&
                          (g_fp32_path == 0 ? (N / 128) * H >= 296 : g_fp32_path == 2);
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.reorder && launch_reorder_queries(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (w.prune && (launch_reorder_keys(a, w) != cudaSuccess || launch_prune_stats(a, w) != cudaSuccess)) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
     const cudaError_t sweep = tc ? launch_score_select_tc(a, w)
                               : tiled32 ? launch_score_select_fp32_tiled(a, w) : launch_score_select_exact(a);

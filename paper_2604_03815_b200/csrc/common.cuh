@@ -32,6 +32,7 @@ struct WorkItem {
     int nrows;   // 1..384 (128 x the query tiles per CTA of the launched configuration)
     int key_lo;  // graph's first row
     int key_hi;  // one past the graph's last row
+    int tile0;   // number of the graph's first 128-key tile in the per-tile statistics (pruned sweep)
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
@@ -42,16 +43,28 @@ struct FwdWorkspace {
     size_t qperm_off;  // bf16 [N, H, d]: Q in the sweep's row order (only when `reorder`)
     size_t perm_off;   // int  [N]: original row of each sweep row
     size_t code_off;   // u16  [N]: locality codes of the query rows
+    // pruned sweep only (all 0 bytes otherwise):
+    size_t kperm_off;   // int   [N]: original key of each sweep position
+    size_t kcode_off;   // u16   [N]: key codes (norm class, nearest pivot), by node
+    size_t kcs_off;     // u16   [N]: the same in sweep order
+    size_t knorm_off;   // float [N]: squared norm of the node's whole key vector
+    size_t gmax_off;    // u32   [G]: bits of each graph's largest squared key norm
+    size_t qnorm_off;   // float [N, H]: norm of each query row's head slice, in sweep order
+    size_t qstat_off;   // float [max_items, 3, H, d+4]: centroid, radius, centroid norm of each item's 128-row query tiles
+    size_t kstat_off;   // float [max_tiles, H, d+4]: centroid, radius, centroid norm, largest norm of each key tile
     size_t total;
     int max_items;
+    int max_tiles;
     bool reorder;      // the sweep runs the rows of large graphs in locality order (reorder.cu)
+    bool prune;        // the sweep skips key tiles that cannot hold a candidate (prune.cu)
 };
 
 constexpr int64_t kReorderMinNodes = 32768;  // below this the extra launches cost more than they can save
 
 // `tc`: the tensor-core sweep will run (bf16 mode and a supported (d, k))
-inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, bool tc) {
+inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, bool tc, bool prune = false) {
     FwdWorkspace w;
+    const int32_t g = G > 0 ? G : 1;
     w.max_items = (int)(N / 128 + (G > 0 ? G : 1) + 1);
     w.items_off = kStatusBytes;
     w.kpack_off = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
@@ -59,7 +72,18 @@ inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t 
     w.qperm_off = align_up(w.kpack_off + (tc ? (size_t)N * H * d * 2 : 0));
     w.perm_off = align_up(w.qperm_off + (w.reorder ? (size_t)N * H * d * 2 : 0));
     w.code_off = align_up(w.perm_off + (w.reorder ? (size_t)N * 4 : 0));
-    w.total = align_up(w.code_off + (w.reorder ? (size_t)N * 2 : 0));
+    w.prune = prune && w.reorder;
+    w.max_tiles = (int)(N / 128 + g + 2);  // tile0 of a graph = floor(first row / 128) + graph index
+    const size_t p = w.prune ? 1 : 0, rec = (size_t)(d + 4) * 4;
+    w.kperm_off = align_up(w.code_off + (w.reorder ? (size_t)N * 2 : 0));
+    w.kcode_off = align_up(w.kperm_off + p * (size_t)N * 4);
+    w.kcs_off = align_up(w.kcode_off + p * (size_t)N * 2);
+    w.knorm_off = align_up(w.kcs_off + p * (size_t)N * 2);
+    w.gmax_off = align_up(w.knorm_off + p * (size_t)N * 4);
+    w.qnorm_off = align_up(w.gmax_off + p * (size_t)g * 4);
+    w.qstat_off = align_up(w.qnorm_off + p * (size_t)N * H * 4);
+    w.kstat_off = align_up(w.qstat_off + p * (size_t)w.max_items * 3 * H * rec);
+    w.total = align_up(w.kstat_off + p * (size_t)w.max_tiles * H * rec);
     return w;
 }
 
@@ -178,6 +202,12 @@ cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_it
 cudaError_t launch_pack_keys(const FwdArgs& a, const FwdWorkspace& w);
 // reorder.cu: locality codes, per-graph bucket sort, row-permuted copy of Q (after launch_plan)
 cudaError_t launch_reorder_queries(const FwdArgs& a, const FwdWorkspace& w);
+// reorder.cu, pruned sweep: keys of large graphs sorted by (norm class, locality code) and regrouped by
+// head in that order (replaces launch_pack_keys; after launch_reorder_queries, which owns the code buffer first)
+cudaError_t launch_reorder_keys(const FwdArgs& a, const FwdWorkspace& w);
+// prune.cu: centroid / radius / norm statistics of every item's query rows and of every key tile
+cudaError_t launch_prune_stats(const FwdArgs& a, const FwdWorkspace& w);
+constexpr int kMinRowsToSort = 8192;  // smaller graphs keep their row and key order
 // score_select_exact.cu: CUDA-core scores + running top-k, any supported (d, k), fp32 or bf16 storage
 cudaError_t launch_score_select_exact(const FwdArgs& a);
 // score_select_tc.cu: tcgen05 scores + running top-k (bf16 storage); returns cudaErrorNotSupported

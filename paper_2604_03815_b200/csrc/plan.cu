@@ -69,6 +69,7 @@ plan_kernel(const int32_t* __restrict__ offs, int G, int N, int rows_per_item, i
                 it.nrows = min(rows_per_item, hi - it.row0);
                 it.key_lo = lo;
                 it.key_hi = hi;
+                it.tile0 = lo / 128 + g;
                 items[base + t] = it;
             }
         }

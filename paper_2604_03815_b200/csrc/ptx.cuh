@@ -229,6 +229,10 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
 __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+// one 8-byte store (a reader's 8-byte load sees both words of one store)
+__device__ __forceinline__ void sts_v2(uint32_t addr, uint32_t x, uint32_t y) {
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
 
 // max of three floats in one instruction (sm_100+)
 __device__ __forceinline__ float max3(float a, float b, float c) {

@@ -34,7 +34,7 @@ template <typename T, int D, int E, bool REGROUPED>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int32_t* __restrict__ offs, int G,
                    int N, int H, int k, int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
-                   const StatusBlock* __restrict__ sb) {
+                   const StatusBlock* __restrict__ sb, const int* __restrict__ kperm) {
     if (sb->status != KMIP_OK) return;
     constexpr int CAP = 32 * E;
     static_assert((sizeof(T) == 2) == REGROUPED, "bf16 keys come regrouped, fp32 keys in place");
@@ -122,7 +122,8 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                 const bool pass = valid[u] && (s > tau);
                 const unsigned m = __ballot_sync(0xFFFFFFFFu, pass);
                 if (m) {
-                    if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, jj[u]);
+                    // pruned sweep: the groups are positions of the sweep's key order; the answer names the keys
+                    if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, kperm ? __ldg(kperm + jj[u]) : jj[u]);
                     cnt += __popc(m);
                     if (cnt > room - 32) {
                         tau = fmaxf(floor_tau, E <= 4 ? warp_merge_row_chunks(row, k, cnt, lane) : warp_compact_row<E>(row, k, cnt, lane));
@@ -138,14 +139,14 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
 }
 
 template <typename T, int D>
-cudaError_t launch_d(const FwdArgs& a, const T* keys) {
+cudaError_t launch_d(const FwdArgs& a, const T* keys, const int* kperm = nullptr) {
     constexpr bool REGROUPED = sizeof(T) == 2;
     const long long n_rows = (long long)a.N * a.H;
     const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
 #define KMIP_LAUNCH_REFINE(E_) \
     refine_topk_kernel<T, D, E_, REGROUPED><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
         static_cast<const T*>(a.Q), keys, a.graph_offsets, a.G, (int)a.N, a.H, a.k, \
-        a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws))
+        a.topk_idx, a.topk_score, reinterpret_cast<const StatusBlock*>(a.ws), kperm)
     // pending room CAP-k: the survivors of a row (rarely more than 2k) should fit without intermediate
     // compactions, and the final sort costs log^2(CAP) compare-exchange stages
     if (a.k <= 16) KMIP_LAUNCH_REFINE(2);
@@ -160,11 +161,12 @@ cudaError_t launch_d(const FwdArgs& a, const T* keys) {
 cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w) {
     using T = __nv_bfloat16;
     const T* keys = reinterpret_cast<const T*>(a.ws + w.kpack_off);
+    const int* kperm = w.prune ? reinterpret_cast<const int*>(a.ws + w.kperm_off) : nullptr;
     switch (a.d) {
-        case 16: return launch_d<T, 16>(a, keys);
-        case 32: return launch_d<T, 32>(a, keys);
-        case 64: return launch_d<T, 64>(a, keys);
-        case 128: return launch_d<T, 128>(a, keys);
+        case 16: return launch_d<T, 16>(a, keys, kperm);
+        case 32: return launch_d<T, 32>(a, keys, kperm);
+        case 64: return launch_d<T, 64>(a, keys, kperm);
+        case 128: return launch_d<T, 128>(a, keys, kperm);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -242,13 +242,49 @@ __device__ __forceinline__ void append_groups(const float (&sub)[16], const floa
     }
 }
 
-template <int D, int KG, int NQT, int S, bool DUMP>
+// What the pruned sweep (PRUNE) adds to the kernel below.  The TMA producer decides, 32 key tiles at a
+// time (one per lane), which tiles no row of the CTA's query block can take a candidate from (bounds of
+// prune.cu against the thresholds the selection warps publish per warp) and loads only the others, so the
+// tiles that flow through the pipeline are no longer numbered consecutively:
+//   * the producer writes each loaded tile's first key into sStageKey[stage] before it arms the stage's
+//     full barrier, and ends an item with a pseudo tile (first key -1, no data, a plain arrive);
+//   * an issuer reads it after the full-barrier wait, acknowledges the read with an arrival of its own on
+//     the stage's empty barrier (with one query tile per CTA an issuer owns no pair of every other tile
+//     and would otherwise read the stage after it was refilled), copies it to sBufKey[buffer] before the
+//     pair's commit (or, for the pseudo tile, a plain arrive on the pair's barrier) and leaves the item
+//     after the pseudo tile;
+//   * a selection warp reads sBufKey[buffer] after its wait and before it hands the buffer back.
+// A skipped tile would have produced no candidate: every group maximum in it is below the row's
+// threshold at decision time, and thresholds only rise.  So the lists are those of the full sweep.
+struct PruneArgs {
+    const float* qstat;  // [items, H, D+4]
+    const float* kstat;  // [tiles, H, D+4]
+    const float* qnorm;  // [N, H], sweep order
+};
+
+constexpr int kEndOfItem = -1;  // "first key" of the pseudo tile that ends an item
+constexpr int kDeadPair = -2;   // "first key" of a (key tile, query tile) pair the bounds ruled out
+
+// A selection warp tells the producer the smallest threshold of its rows and the smallest
+// threshold / |q| (only rows with a positive threshold can use the norm bound), tagged with the item.
+__device__ __forceinline__ void publish_thresholds(float tau, float inv_qn, int ic, uint32_t stat_s, int lane) {
+    const float ratio = tau > 0.0f ? tau * inv_qn : -CUDART_INF_F;  // rows past the item's end have tau = +inf
+    const uint32_t tm = __reduce_min_sync(FULL, order_bits(tau));
+    const uint32_t rm = __reduce_min_sync(FULL, order_bits(ratio));
+    if (lane == 0) {
+        ptx::sts_v2(stat_s, (uint32_t)ic, __float_as_uint(unorder_bits(tm)));
+        ptx::sts_v2(stat_s + 8u, (uint32_t)ic, __float_as_uint(unorder_bits(rm)));
+    }
+}
+
+template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE>
 __global__ void __launch_bounds__(NQT * 128 + 96, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
                        float* __restrict__ dump, int dump_ld /* = N */, int dbg_arg, long long* __restrict__ timing,
-                       long long wait_limit, int drop_first_tile, const int* __restrict__ perm) {
+                       long long wait_limit, int drop_first_tile, const int* __restrict__ perm, const PruneArgs pr) {
+    static_assert(!(DUMP && PRUNE), "the score dump sweeps every tile");
     const int dbg = kSweepDebug ? dbg_arg : 0;
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
@@ -266,6 +302,11 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     uint32_t* sTmem = reinterpret_cast<uint32_t*>(sBars + Sp::NBARS);
     volatile int* sAbort = reinterpret_cast<volatile int*>(sTmem + 1);
     volatile int* sFlushReq = reinterpret_cast<volatile int*>(sTmem + 2);  // CTA-wide flush request counter
+    volatile int* sStageKey = reinterpret_cast<volatile int*>(sTmem + 4);   // [4] first key of the tile in a key stage
+    volatile int* sBufKey = reinterpret_cast<volatile int*>(sTmem + 8);     // [4] first key of the pair in an accumulator buffer
+    // [warp][2] {item number, float bits}: smallest threshold and smallest threshold / query norm of the warp's rows
+    const uint32_t warp_stat_s = ptx::smem_u32(sTmem + 12);
+    volatile int* sStageDead = reinterpret_cast<volatile int*>(sTmem + 60);  // [4] query tiles that skip the stage's key tile (bit mask)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     Bars bars{ptx::smem_u32(sBars), S, NQT};
@@ -276,7 +317,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         ptx::mbar_init(bars.done(), NISS);
         for (int s = 0; s < S; ++s) {
             ptx::mbar_init(bars.k_full(s), 1);
-            ptx::mbar_init(bars.k_empty(s), NQT);  // one arrival per query tile
+            ptx::mbar_init(bars.k_empty(s), NQT + (PRUNE ? NISS : 0));  // one arrival per query tile (and per issuer's read)
         }
         for (int b = 0; b < NBUF; ++b) {
             for (int q = 0; q < NQT; ++q) ptx::mbar_init(bars.t_full(b, q), 1);
@@ -284,6 +325,8 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
         *sAbort = 0;
         *sFlushReq = 0;
+        if (PRUNE)
+            for (int i = 0; i < 2 * NEPI; ++i) ptx::sts_v2(warp_stat_s + 8u * i, 0xFFFFFFFFu, 0u);  // item number -1: not valid
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -303,7 +346,127 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const int n_items = sb->n_items;
     const long long total = (long long)n_items * H;
 
-    if (warp == NEPI) {
+    if (PRUNE && warp == NEPI) {
+        // ------------------------------------------------------------------ TMA producer, pruned sweep
+        // All 32 lanes evaluate bounds (one tile each); lane 0 runs the pipeline.
+        constexpr int REC = D + 4;
+        int kt = 0, ic = 0;
+        bool ok = true;
+        for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
+            const int h = (int)(w / n_items);
+            const int item = (int)(w % n_items);
+            const WorkItem it = items[item];
+            if (lane == 0) {
+                ok = wait_or_abort<kRelaxedPollNs>(bars.q_empty(), (ic & 1) ^ 1, sAbort, sb, 1, wait_limit);
+                if (ok) {
+                    ptx::mbar_arrive_expect_tx(bars.q_full(), NQT * Sh::TILE_BYTES);
+                    for (int qt = 0; qt < NQT; ++qt)
+                        for (int ch = 0; ch < Sh::KCH; ++ch)
+                            ptx::tma_load_2d(ptx::smem_u32(sQ + qt * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmQ,
+                                             h * D + ch * 64, it.row0 + qt * BM, bars.q_full());
+                }
+            }
+            ok = __shfl_sync(FULL, (int)ok, 0) != 0;
+            if (!ok) break;
+            // one record per 128-row query tile of the item: centroid, radius, centroid norm (all lanes read
+            // the same addresses); the first record also holds the tile the sweep starts at
+            const float* qrec0 = pr.qstat + ((size_t)item * NQT * H + h) * REC;
+            const int nq = (it.nrows + BM - 1) / BM;  // query tiles that hold rows
+            const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
+            // The sweep starts at the tile the statistics kernel chose for the block, runs to the end of the
+            // graph and then takes the tiles in front of the start.
+            const int jstart = min(max(__float_as_int(__ldg(qrec0 + D + 3)), 0), ntiles - 1);
+            for (int seg = 0; ok && seg < 2; ++seg) {
+                const int seg_hi = seg == 0 ? ntiles : jstart;
+                for (int j0 = seg == 0 ? jstart : 0; ok && j0 < seg_hi; j0 += 32) {
+                    const int j = j0 + lane;
+                    unsigned dead = (1u << NQT) - 1u;  // query tiles that cannot take a candidate from key tile j
+                    bool rest_dead = false;
+                    if (j < seg_hi) {
+                        const float4* krec = reinterpret_cast<const float4*>(pr.kstat + ((size_t)(it.tile0 + j) * H + h) * REC);
+                        float4 ck[D / 4];
+#pragma unroll
+                        for (int c = 0; c < D / 4; ++c) ck[c] = __ldg(krec + c);
+                        const float4 ktail = __ldg(krec + D / 4);
+                        const float r_t = ktail.x, n_ct = ktail.y, k_max = ktail.z, k_max_rest = ktail.w;
+                        rest_dead = true;
+#pragma unroll
+                        for (int qt = 0; qt < NQT; ++qt) {
+                            if (qt >= nq) continue;  // no rows: nothing to object
+                            const float4* qrec = reinterpret_cast<const float4*>(qrec0 + (size_t)qt * H * REC);
+                            float dot = 0.0f;
+#pragma unroll
+                            for (int c = 0; c < D / 4; ++c) {
+                                const float4 t = __ldg(qrec + c);
+                                dot = fmaf(ck[c].x, t.x, dot); dot = fmaf(ck[c].y, t.y, dot);
+                                dot = fmaf(ck[c].z, t.z, dot); dot = fmaf(ck[c].w, t.w, dot);
+                            }
+                            const float4 qtail = __ldg(qrec + D / 4);
+                            const float r_b = qtail.x, n_cq = qtail.y;
+                            const float spread = n_cq * r_t + n_ct * r_b + r_b * r_t;
+                            // rounding of the bound itself and of the tensor-core scores, both relative to |q| |k|
+                            const float bound = dot + spread + 1e-4f * (n_cq * n_ct + spread);
+                            // thresholds published for THIS item; a warp that has not started it yet counts as -inf
+                            float tau_min = CUDART_INF_F, ratio_min = CUDART_INF_F;
+#pragma unroll
+                            for (int wq = 4 * qt; wq < 4 * qt + 4; ++wq) {
+                                const uint2 a = ptx::lds_v2(warp_stat_s + 16u * wq);
+                                const uint2 b = ptx::lds_v2(warp_stat_s + 16u * wq + 8u);
+                                tau_min = fminf(tau_min, (int)a.x == ic ? __uint_as_float(a.y) : -CUDART_INF_F);
+                                ratio_min = fminf(ratio_min, (int)b.x == ic ? __uint_as_float(b.y) : -CUDART_INF_F);
+                            }
+                            if (!(bound < tau_min || k_max < ratio_min)) dead &= ~(1u << qt);
+                            rest_dead = rest_dead && k_max_rest < ratio_min;  // this key tile and every later one of the graph
+                        }
+                    }
+                    const unsigned skip_mask = __ballot_sync(FULL, dead == (1u << NQT) - 1u);
+                    const bool seg_done = __any_sync(FULL, rest_dead);
+                    const int nb = min(32, seg_hi - j0);
+                    for (int l = 0; l < nb; ++l) {
+                        const unsigned dead_l = __shfl_sync(FULL, dead, l);
+                        if (lane != 0 || ((skip_mask >> l) & 1u) || !ok) continue;
+                        const int s = kt % S;
+                        if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit))) continue;
+                        const int key0 = it.key_lo + (j0 + l) * BN;
+                        sStageKey[s] = key0;
+                        sStageDead[s] = (int)dead_l;
+                        ptx::mbar_arrive_expect_tx(bars.k_full(s), Sh::TILE_BYTES);
+                        for (int ch = 0; ch < Sh::KCH; ++ch)
+                            ptx::tma_load_2d(ptx::smem_u32(sK + s * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmK,
+                                             ch * 64, h * dump_ld + key0, bars.k_full(s));
+                        ++kt;
+                    }
+                    ok = __shfl_sync(FULL, (int)ok, 0) != 0;
+                    kt = __shfl_sync(FULL, kt, 0);
+                    if (seg_done) break;  // the lanes after the first dead one were skipped by the same test
+                }
+            }
+            if (!ok) break;
+            if (lane == 0) {
+                // the pseudo tile that ends the item: no data, the phase completes with this arrive
+                const int s = kt % S;
+                ok = wait_or_abort<kRelaxedPollNs>(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit);
+                if (ok) {
+                    sStageKey[s] = kEndOfItem;
+                    ptx::mbar_arrive(bars.k_full(s));
+                    ++kt;
+                }
+            }
+            ok = __shfl_sync(FULL, (int)ok, 0) != 0;
+            kt = __shfl_sync(FULL, kt, 0);
+            ++ic;
+        }
+        if (!ok && lane == 0) {
+            // give copies that are still in flight a bounded time to land before the CTA exits; a stage
+            // whose last use was a pseudo tile has completed that phase already
+            const long long t0 = clock64();
+            for (int s = 0; s < S && kt > 0; ++s) {
+                const int last = kt - 1 - ((kt - 1 - s) % S + S) % S;
+                if (last < 0) continue;
+                while (!ptx::mbar_try_wait(bars.k_full(s), (last / S) & 1) && clock64() - t0 < 40000000ll) {}
+            }
+        }
+    } else if (warp == NEPI) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             int kt = 0, ic = 0;
@@ -371,7 +534,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 if (!(ok = wait_or_abort<0>(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
                 ptx::tc_fence_after();
                 const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
-                for (int j = 0; ok && j < ntiles; ++j, ++kt) {
+                for (int j = 0; ok && (PRUNE || j < ntiles); ++j, ++kt) {
                     const int s = kt % S;
                     const uint64_t stage_off = (uint64_t)((s * Sh::TILE_BYTES) >> 4);  // start-address field counts 16-byte units
                     // Both issuers wait for EVERY key tile, also one whose pairs all belong to the other
@@ -381,6 +544,12 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     long long c0 = (dbg & 8) ? clock64() : 0;
                     if (!(ok = wait_or_abort<0>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
                     if (dbg & 8) w_kfull += clock64() - c0;
+                    int tile_key = 0, tile_dead = 0;
+                    if constexpr (PRUNE) {
+                        tile_key = sStageKey[s];
+                        tile_dead = sStageDead[s];
+                        ptx::mbar_arrive(bars.k_empty(s));  // the read is done: one of the arrivals the refill waits for
+                    }
 #pragma unroll
                     for (int qt = 0; qt < NQT; ++qt) {
                         const int seq = kt * NQT + qt;
@@ -390,6 +559,17 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         if (!(ok = wait_or_abort<0>(bars.t_empty(b), ((seq >> 2) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
                         if (dbg & 8) w_tempty += clock64() - c1;
                         ptx::tc_fence_after();
+                        if constexpr (PRUNE) {
+                            // a pair without scores (end of item, or ruled out for this query tile) still takes
+                            // its turn in the ring, so that the buffers and barrier phases stay in step
+                            const bool no_scores = tile_key == kEndOfItem || ((tile_dead >> qt) & 1);
+                            sBufKey[b] = tile_key == kEndOfItem ? kEndOfItem : no_scores ? kDeadPair : tile_key;
+                            __threadfence_block();
+                            if (no_scores) {
+                                ptx::mbar_arrive(bars.t_full(b, qt));
+                                continue;
+                            }
+                        }
                         if (qt < nq) {
                             const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
 #pragma unroll
@@ -397,6 +577,10 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                                 ptx::mma_bf16_ss(d_tmem, desc_q[qt][ks], desc_k0[ks] + stage_off, kInstrDesc, ks > 0 ? 1u : 0u);
                         }
                         ptx::mma_commit(bars.t_full(b, qt));
+                    }
+                    if (PRUNE && ok && tile_key == kEndOfItem) {
+                        ++kt;
+                        break;
                     }
                 }
                 if (!ok) break;
@@ -427,7 +611,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16);  // buffer 0, this warp's lanes
         RowSel<KG> rs;
         int flush_seen = 0;
-        int tcnt = 0;
+        int tcnt = 0, ic = 0;
         bool ok = true;
         long long w_tfull = 0, t_work = 0, t_begin = clock64();
         long long prof[4] = {0, 0, 0, 0};
@@ -439,6 +623,13 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const bool rvalid = local < it.nrows;
             if (active) row_init<KG>(rs, wl, k, lane, rvalid);
             __syncwarp();
+            float inv_qn = 1.0f;
+            if constexpr (PRUNE) {
+                // nothing can be skipped for this warp's rows until a flush has raised their thresholds;
+                // a warp without rows never objects
+                if (active && rvalid) inv_qn = 1.0f / fmaxf(__ldg(pr.qnorm + (size_t)(it.row0 + local) * H + h), 1e-30f);
+                publish_thresholds(active ? rs.tau : CUDART_INF_F, inv_qn, ic, warp_stat_s + 16u * warp, lane);
+            }
             const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;
             // This warp group's (key tile, query tile) pair is number tcnt*NQT + qt of the CTA; its buffer
             // is that number mod 4, and the (buffer, query tile) barrier has been used tcnt >> kUseShift
@@ -447,12 +638,13 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (DUMP || !active) {
                 // debug dump of the raw scores, or a query tile past the item's rows that only keeps
                 // the barriers in step
-                for (int j = 0; j < ntiles; ++j, ++tcnt) {
+                for (int j = 0; PRUNE || j < ntiles; ++j, ++tcnt) {
                     const int b = (tcnt * NQT + qt) & (NBUF - 1);
                     ok = wait_or_abort(full_bar0 + (uint32_t)b * (8u * NQT), (uint32_t)(tcnt >> kUseShift) & 1u, sAbort, sb,
                                        6, wait_limit);
                     ok = __all_sync(FULL, ok);
                     if (!ok) break;
+                    const int tile_key = PRUNE ? sBufKey[b] : 0;
                     if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
                     ptx::tc_fence_after();
                     if (DUMP && active) {
@@ -473,11 +665,15 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
+                    if (PRUNE && tile_key == kEndOfItem) {
+                        ++tcnt;
+                        break;
+                    }
                 }
             } else {
                 const int ragged_j = ((it.key_hi - it.key_lo) & (BN - 1)) ? ntiles - 1 : -1;  // only the last tile can be short
                 int key0 = it.key_lo;
-                for (int j = 0; j < ntiles; ++j, ++tcnt, key0 += BN) {
+                for (int j = 0; PRUNE || j < ntiles; ++j, ++tcnt, key0 += BN) {
                     const int b = (tcnt * NQT + qt) & (NBUF - 1);
                     const uint32_t full_bar = full_bar0 + (uint32_t)b * (8u * NQT);
                     const uint32_t full_par = (uint32_t)(tcnt >> kUseShift) & 1u;
@@ -486,18 +682,29 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         // The scores are still not there after the try's own (hardware-bounded) wait:
                         // merge pending candidates into the lists meanwhile (always allowed, and it
                         // raises the thresholds early), then block.
-                        if (!(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
+                        if (!(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) {
+                            flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
+                            if constexpr (PRUNE) publish_thresholds(rs.tau, inv_qn, ic, warp_stat_s + 16u * warp, lane);
+                        }
                         ok = wait_or_abort(full_bar, full_par, sAbort, sb, 6, wait_limit);
                         ok = __all_sync(FULL, ok);
                         if (!ok) break;
                     }
                     const long long c1 = (dbg & 8) ? clock64() : 0;
+                    if constexpr (PRUNE) key0 = sBufKey[b];  // the tiles that arrive are not consecutive
                     // this query tile's MMAs on the key tile have retired; once that holds for every query
                     // tile the key stage can be refilled
                     if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
+                    if (PRUNE && key0 < 0) {
+                        __syncwarp();  // every lane has read the buffer's key
+                        if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
+                        if (key0 == kDeadPair) continue;  // no scores for this query tile; the next pair follows
+                        ++tcnt;
+                        break;
+                    }
                     ptx::tc_fence_after();
                     const uint32_t taddr = taddr0 + (uint32_t)(b * BN);
-                    const bool ragged = j == ragged_j;
+                    const bool ragged = PRUNE ? key0 + BN > it.key_hi : j == ragged_j;
                     const int ncol = it.key_hi - key0;  // columns that exist; below 128 only in a ragged tile
                     // two 64-column halves keep the register footprint small; the accumulator buffer
                     // goes back to the MMA issuers as soon as the second half is in registers
@@ -536,6 +743,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                             if (do_flush) {
                                 const long long p1 = (dbg & 8) ? clock64() : 0;
                                 flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
+                                if constexpr (PRUNE) publish_thresholds(rs.tau, inv_qn, ic, warp_stat_s + 16u * warp, lane);
                                 flush_seen = req + ((req == flush_seen) ? 1 : 0);
                                 if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
                             }
@@ -566,6 +774,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 }
                 __syncwarp();
             }
+            ++ic;
         }
         if ((dbg & 8) && timing && threadIdx.x == 0) {
             timing[blockIdx.x * 8 + 4] = clock64() - t_begin;
@@ -637,18 +846,22 @@ int sm_count() {
     return sms[dev];
 }
 
-template <int D, int KG, int NQT, int S, bool DUMP>
+template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE>
 cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
     constexpr size_t smem_bytes = 1024 + (size_t)(NQT + S) * Sh::TILE_BYTES + (size_t)NQT * 128 * Sp::SLOTS * 8 +
-                                  (size_t)Sp::NBARS * 8 + 16 + 64;
+                                  (size_t)Sp::NBARS * 8 + 16 + 240;
     static_assert(smem_bytes <= 232448, "shared memory budget of one CTA");
     CUtensorMap tmQ, tmK;
     if (!make_tensor_map<D>(&tmQ, w.reorder ? static_cast<const void*>(a.ws + w.qperm_off) : a.Q, a.N, (int64_t)a.H * D) ||
         !make_tensor_map<D>(&tmK, a.ws + w.kpack_off, a.N * a.H, D))
         return cudaErrorInvalidValue;
-    auto kern = score_select_tc_kernel<D, KG, NQT, S, DUMP>;
+    auto kern = score_select_tc_kernel<D, KG, NQT, S, DUMP, PRUNE>;
+    PruneArgs pr{nullptr, nullptr, nullptr};
+    if (PRUNE)
+        pr = PruneArgs{reinterpret_cast<const float*>(a.ws + w.qstat_off), reinterpret_cast<const float*>(a.ws + w.kstat_off),
+                       reinterpret_cast<const float*>(a.ws + w.qnorm_off)};
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (err != cudaSuccess) return err;
     const long long max_total = (long long)w.max_items * a.H;
@@ -656,34 +869,34 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
         a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing, g_wait_limit_cycles,
-        g_drop_first_tile, (w.reorder && !DUMP) ? reinterpret_cast<const int*>(a.ws + w.perm_off) : nullptr);
+        g_drop_first_tile, (w.reorder && !DUMP) ? reinterpret_cast<const int*>(a.ws + w.perm_off) : nullptr, pr);
     return cudaGetLastError();
 }
 
-template <int D, bool DUMP>
+template <int D, bool DUMP, bool PRUNE>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     // (list groups KG, query tiles per CTA, key stages) by k and head width; shared memory decides
     if (a.k <= 32) {
-        if constexpr (D <= 32) return launch_cfg<D, 4, 3, 4, DUMP>(a, w, dump);
-        else if constexpr (D == 64) return launch_cfg<D, 4, 2, 3, DUMP>(a, w, dump);
-        else return launch_cfg<D, 4, 1, 3, DUMP>(a, w, dump);
+        if constexpr (D <= 32) return launch_cfg<D, 4, 3, 4, DUMP, PRUNE>(a, w, dump);
+        else if constexpr (D == 64) return launch_cfg<D, 4, 2, 3, DUMP, PRUNE>(a, w, dump);
+        else return launch_cfg<D, 4, 1, 3, DUMP, PRUNE>(a, w, dump);
     }
     if (a.k <= 64) {
-        if constexpr (D <= 32) return launch_cfg<D, 8, 2, 3, DUMP>(a, w, dump);
-        else if constexpr (D == 64) return launch_cfg<D, 8, 1, 4, DUMP>(a, w, dump);
-        else return launch_cfg<D, 8, 1, 3, DUMP>(a, w, dump);
+        if constexpr (D <= 32) return launch_cfg<D, 8, 2, 3, DUMP, PRUNE>(a, w, dump);
+        else if constexpr (D == 64) return launch_cfg<D, 8, 1, 4, DUMP, PRUNE>(a, w, dump);
+        else return launch_cfg<D, 8, 1, 3, DUMP, PRUNE>(a, w, dump);
     }
-    if constexpr (D <= 64) return launch_cfg<D, 16, 1, 3, DUMP>(a, w, dump);
+    if constexpr (D <= 64) return launch_cfg<D, 16, 1, 3, DUMP, PRUNE>(a, w, dump);
     else return cudaErrorNotSupported;
 }
 
-template <bool DUMP>
+template <bool DUMP, bool PRUNE>
 cudaError_t launch_any(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     switch (a.d) {
-        case 16: return launch_d<16, DUMP>(a, w, dump);
-        case 32: return launch_d<32, DUMP>(a, w, dump);
-        case 64: return launch_d<64, DUMP>(a, w, dump);
-        case 128: return launch_d<128, DUMP>(a, w, dump);
+        case 16: return launch_d<16, DUMP, PRUNE>(a, w, dump);
+        case 32: return launch_d<32, DUMP, PRUNE>(a, w, dump);
+        case 64: return launch_d<64, DUMP, PRUNE>(a, w, dump);
+        case 128: return launch_d<128, DUMP, PRUNE>(a, w, dump);
         default: return cudaErrorNotSupported;
     }
 }
@@ -714,13 +927,13 @@ int score_select_tc_rows_per_item(int32_t d, int32_t k) {  // 128 * query tiles 
 }  // 128 * query tiles per CTA
 
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w) {
-    return launch_any<false>(a, w, nullptr);
+    return w.prune ? launch_any<false, true>(a, w, nullptr) : launch_any<false, false>(a, w, nullptr);
 }
 
 // Test hook: same TMA / tcgen05 pipeline, but the selection warps write every score of the tile to
 // dump[h][i][j] (ld = N) instead of filtering.  Only for small single problems.
 cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
-    return launch_any<true>(a, w, dump);
+    return launch_any<true, false>(a, w, dump);
 }
 
 }  // namespace kmip
