@@ -209,6 +209,15 @@ def kmip_debug_tc_scores(Q, K, scores, workspace, stream=None) -> int:
 # ------------------------------------------------------------------------------------------------
 # Buffer helpers (allocation only)
 # ------------------------------------------------------------------------------------------------
+def sweep_counters(buf) -> None:
+    """Diagnostic hook (not in kmip.h): int64 device tensor of 8 * SMs entries that the pruned sweep fills
+    per CTA with {key tiles, tiles loaded, (key tile, query tile) pairs, pairs scored}; None switches it off."""
+    f = lib().kmip_debug_set_timing
+    f.argtypes = [ctypes.c_void_p]
+    f.restype = None
+    f(ctypes.c_void_p(buf.data_ptr()) if buf is not None else ctypes.c_void_p(0))
+
+
 def storage_dtype(mode: int):
     return torch.float32 if mode == KMIP_FP32_EXACT else torch.bfloat16
 

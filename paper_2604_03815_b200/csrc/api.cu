@@ -233,6 +233,9 @@ void kmip_debug_fp32_path(int which) { g_fp32_path = which; }
 
 // ---- timing experiments (not part of kmip.h): see set_score_select_debug_flags
 void kmip_debug_set_flags(int flags) { set_score_select_debug_flags(flags); }
+// buf: device array of 8 * (number of SMs) int64, or NULL to switch off.  The pruned sweep writes, per CTA,
+// {key tiles of its work items, tiles it loaded (end-of-item markers included), (key tile, query tile)
+// pairs, pairs it scored}; debug builds of the full sweep write cycle counters there.
 void kmip_debug_set_timing(void* buf) { set_score_select_debug_timing(static_cast<long long*>(buf)); }
 
 // ---- test hook (not part of kmip.h): makes one bounded device-side wait run out, see score_select_tc.cu

@@ -10,6 +10,9 @@
 // result back to the row's own place; nothing else sees the permutation.  On point-cloud-like data
 // (queries in tight clusters) this removes about a tenth of the sweep time; on unstructured data
 // it changes nothing.
+//
+// The pruned sweep (prune.cu) also orders the KEYS of large graphs, by (norm class, nearest pivot), and
+// takes the query codes from the same pivots; see pivot_code_kernel below.
 #include <algorithm>
 
 #include "common.cuh"

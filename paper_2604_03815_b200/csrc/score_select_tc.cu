@@ -352,6 +352,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         constexpr int REC = D + 4;
         int kt = 0, ic = 0;
         bool ok = true;
+        long long n_all = 0, n_pairs_all = 0, n_pairs_live = 0;  // counters for the optional statistics buffer
         for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
             const int h = (int)(w / n_items);
             const int item = (int)(w % n_items);
@@ -376,6 +377,8 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             // The sweep starts at the tile the statistics kernel chose for the block, runs to the end of the
             // graph and then takes the tiles in front of the start.
             const int jstart = min(max(__float_as_int(__ldg(qrec0 + D + 3)), 0), ntiles - 1);
+            n_all += ntiles;
+            n_pairs_all += (long long)ntiles * nq;
             for (int seg = 0; ok && seg < 2; ++seg) {
                 const int seg_hi = seg == 0 ? ntiles : jstart;
                 for (int j0 = seg == 0 ? jstart : 0; ok && j0 < seg_hi; j0 += 32) {
@@ -430,6 +433,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         const int key0 = it.key_lo + (j0 + l) * BN;
                         sStageKey[s] = key0;
                         sStageDead[s] = (int)dead_l;
+                        n_pairs_live += nq - __popc(dead_l & ((1u << nq) - 1u));
                         ptx::mbar_arrive_expect_tx(bars.k_full(s), Sh::TILE_BYTES);
                         for (int ch = 0; ch < Sh::KCH; ++ch)
                             ptx::tma_load_2d(ptx::smem_u32(sK + s * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmK,
@@ -455,6 +459,12 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ok = __shfl_sync(FULL, (int)ok, 0) != 0;
             kt = __shfl_sync(FULL, kt, 0);
             ++ic;
+        }
+        if (timing && lane == 0) {  // per CTA: key tiles of its items, tiles loaded (with the end markers), pairs, pairs scored
+            timing[blockIdx.x * 8 + 0] = n_all;
+            timing[blockIdx.x * 8 + 1] = kt;
+            timing[blockIdx.x * 8 + 2] = n_pairs_all;
+            timing[blockIdx.x * 8 + 3] = n_pairs_live;
         }
         if (!ok && lane == 0) {
             // give copies that are still in flight a bounded time to land before the CTA exits; a stage

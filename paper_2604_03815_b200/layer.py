@@ -60,10 +60,12 @@ class KMIPSelfAttention(torch.nn.Module):
     d_head must be 16, 32, 64 or 128 and k <= 128.  dtype bfloat16 selects the tensor-core mode,
     float32 the fp32 mode.  attn_dropout is the dropout rate on the k attention weights, active in
     training mode only (the paper's graph models use 0.5); every forward call draws a fresh seed
-    from torch's CPU generator, so torch.manual_seed makes a run repeatable."""
+    from torch's CPU generator, so torch.manual_seed makes a run repeatable.  prune=True selects the
+    tensor-core mode with exact tile skipping (same results, faster on clustered or heavy-tailed keys).
+    set_k changes k between calls (the paper's Sec. 6 suggests annealing k during training)."""
 
     def __init__(self, d_model, num_heads, d_head, k, dtype=torch.bfloat16, device="cuda", bias=False,
-                 attn_dropout=0.0):
+                 attn_dropout=0.0, prune=False):
         super().__init__()
         if dtype not in (torch.bfloat16, torch.float32):
             raise ValueError("dtype must be torch.bfloat16 or torch.float32")
@@ -71,7 +73,9 @@ class KMIPSelfAttention(torch.nn.Module):
         if not 0.0 <= attn_dropout < 1.0:
             raise ValueError("attn_dropout must be in [0, 1)")
         self.attn_dropout = float(attn_dropout)
-        self.mode = kb.KMIP_BF16_TC if dtype == torch.bfloat16 else kb.KMIP_FP32_EXACT
+        if prune and dtype != torch.bfloat16:
+            raise ValueError("prune needs dtype bfloat16 (it is a variant of the tensor-core mode)")
+        self.mode = (kb.KMIP_BF16_TC_PRUNED if prune else kb.KMIP_BF16_TC) if dtype == torch.bfloat16 else kb.KMIP_FP32_EXACT
         inner = num_heads * d_head
         self.w_q = torch.nn.Linear(d_model, inner, bias=bias, device=device, dtype=dtype)
         self.w_k = torch.nn.Linear(d_model, inner, bias=bias, device=device, dtype=dtype)
@@ -79,6 +83,11 @@ class KMIPSelfAttention(torch.nn.Module):
         self.w_o = torch.nn.Linear(inner, d_model, bias=bias, device=device, dtype=dtype)
         for lin in (self.w_q, self.w_k, self.w_v, self.w_o):
             torch.nn.init.normal_(lin.weight, std=1.0 / math.sqrt(lin.in_features))
+
+    def set_k(self, k):
+        if not 1 <= int(k) <= 128:
+            raise ValueError("k must be in 1..128")
+        self.k = int(k)
 
     def forward(self, x, graph_offsets=None, return_indices=False):
         N = x.shape[0]
