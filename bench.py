@@ -284,7 +284,7 @@ def run_ours(args, w):
     # The pruned mode (exact tile skipping) on the same inputs: an extra, reported beside the headline,
     # which stays the full sweep - its tensor-pipe fraction is only meaningful when every score is computed.
     pruned = None
-    if w.mode == wl.MODE_BF16_TC and w.N >= 32768:
+    if w.mode == wl.MODE_BF16_TC and w.N >= 32768 and not args.no_pruned:
         pm = kb.KMIP_BF16_TC_PRUNED
         fbp = kb.ForwardBuffers(w.N, w.G, w.H, w.d, w.k, pm, dev)
 
@@ -413,6 +413,7 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload number (1-5); the headline is 4")
     ap.add_argument("--nodes", type=int, default=0, help="override the node count of configs 3/4 (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-pruned", action="store_true", help="skip the extra measurement of the pruned mode")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

@@ -262,6 +262,7 @@ struct PruneArgs {
     const float* qnorm;  // [N, H], sweep order
 };
 
+constexpr int kPruneTilesPerLane = 1;  // key tiles a producer lane decides per batch (4: staler thresholds, 4 % slower)
 constexpr int kEndOfItem = -1;  // "first key" of the pseudo tile that ends an item
 constexpr int kDeadPair = -2;   // "first key" of a (key tile, query tile) pair the bounds ruled out
 
@@ -379,70 +380,91 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const int jstart = min(max(__float_as_int(__ldg(qrec0 + D + 3)), 0), ntiles - 1);
             n_all += ntiles;
             n_pairs_all += (long long)ntiles * nq;
+            // query tiles (bit mask) that cannot take a candidate from key tile j; `rest` is set when that holds
+            // for tile j and every later tile of the graph by the norm bound alone
+            auto evaluate = [&](int j, bool& rest) -> unsigned {
+                unsigned dead = (1u << NQT) - 1u;
+                const float4* krec = reinterpret_cast<const float4*>(pr.kstat + ((size_t)(it.tile0 + j) * H + h) * REC);
+                float4 ck[D / 4];
+#pragma unroll
+                for (int c = 0; c < D / 4; ++c) ck[c] = __ldg(krec + c);
+                const float4 ktail = __ldg(krec + D / 4);
+                const float r_t = ktail.x, n_ct = ktail.y, k_max = ktail.z, k_max_rest = ktail.w;
+                rest = true;
+#pragma unroll
+                for (int qt = 0; qt < NQT; ++qt) {
+                    if (qt >= nq) continue;  // no rows: nothing to object
+                    const float4* qrec = reinterpret_cast<const float4*>(qrec0 + (size_t)qt * H * REC);
+                    float dot = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < D / 4; ++c) {
+                        const float4 t = __ldg(qrec + c);
+                        dot = fmaf(ck[c].x, t.x, dot); dot = fmaf(ck[c].y, t.y, dot);
+                        dot = fmaf(ck[c].z, t.z, dot); dot = fmaf(ck[c].w, t.w, dot);
+                    }
+                    const float4 qtail = __ldg(qrec + D / 4);
+                    const float r_b = qtail.x, n_cq = qtail.y;
+                    const float spread = n_cq * r_t + n_ct * r_b + r_b * r_t;
+                    // rounding of the bound itself and of the tensor-core scores, both relative to |q| |k|
+                    const float bound = dot + spread + 1e-4f * (n_cq * n_ct + spread);
+                    // thresholds published for THIS item; a warp that has not started it yet counts as -inf
+                    float tau_min = CUDART_INF_F, ratio_min = CUDART_INF_F;
+#pragma unroll
+                    for (int wq = 4 * qt; wq < 4 * qt + 4; ++wq) {
+                        const uint2 a = ptx::lds_v2(warp_stat_s + 16u * wq);
+                        const uint2 b = ptx::lds_v2(warp_stat_s + 16u * wq + 8u);
+                        tau_min = fminf(tau_min, (int)a.x == ic ? __uint_as_float(a.y) : -CUDART_INF_F);
+                        ratio_min = fminf(ratio_min, (int)b.x == ic ? __uint_as_float(b.y) : -CUDART_INF_F);
+                    }
+                    if (!(bound < tau_min || k_max < ratio_min)) dead &= ~(1u << qt);
+                    rest = rest && k_max_rest < ratio_min;
+                }
+                return dead;
+            };
+            // Decisions are taken for a batch of tiles at a time (lane l: tiles l, l + 32, ...) and the batch
+            // is then fed to the pipeline by lane 0; the first batch of an item is small because nothing can
+            // be skipped before the first thresholds exist.
+            constexpr int U = kPruneTilesPerLane;
+            bool first_batch = true;
             for (int seg = 0; ok && seg < 2; ++seg) {
                 const int seg_hi = seg == 0 ? ntiles : jstart;
-                for (int j0 = seg == 0 ? jstart : 0; ok && j0 < seg_hi; j0 += 32) {
-                    const int j = j0 + lane;
-                    unsigned dead = (1u << NQT) - 1u;  // query tiles that cannot take a candidate from key tile j
-                    bool rest_dead = false;
-                    if (j < seg_hi) {
-                        const float4* krec = reinterpret_cast<const float4*>(pr.kstat + ((size_t)(it.tile0 + j) * H + h) * REC);
-                        float4 ck[D / 4];
+                for (int j0 = seg == 0 ? jstart : 0; ok && j0 < seg_hi;) {
+                    const int nbatch = min(first_batch ? 32 : 32 * U, seg_hi - j0);
+                    first_batch = false;
+                    unsigned dead[U];
+                    bool seg_done = false;
 #pragma unroll
-                        for (int c = 0; c < D / 4; ++c) ck[c] = __ldg(krec + c);
-                        const float4 ktail = __ldg(krec + D / 4);
-                        const float r_t = ktail.x, n_ct = ktail.y, k_max = ktail.z, k_max_rest = ktail.w;
-                        rest_dead = true;
-#pragma unroll
-                        for (int qt = 0; qt < NQT; ++qt) {
-                            if (qt >= nq) continue;  // no rows: nothing to object
-                            const float4* qrec = reinterpret_cast<const float4*>(qrec0 + (size_t)qt * H * REC);
-                            float dot = 0.0f;
-#pragma unroll
-                            for (int c = 0; c < D / 4; ++c) {
-                                const float4 t = __ldg(qrec + c);
-                                dot = fmaf(ck[c].x, t.x, dot); dot = fmaf(ck[c].y, t.y, dot);
-                                dot = fmaf(ck[c].z, t.z, dot); dot = fmaf(ck[c].w, t.w, dot);
-                            }
-                            const float4 qtail = __ldg(qrec + D / 4);
-                            const float r_b = qtail.x, n_cq = qtail.y;
-                            const float spread = n_cq * r_t + n_ct * r_b + r_b * r_t;
-                            // rounding of the bound itself and of the tensor-core scores, both relative to |q| |k|
-                            const float bound = dot + spread + 1e-4f * (n_cq * n_ct + spread);
-                            // thresholds published for THIS item; a warp that has not started it yet counts as -inf
-                            float tau_min = CUDART_INF_F, ratio_min = CUDART_INF_F;
-#pragma unroll
-                            for (int wq = 4 * qt; wq < 4 * qt + 4; ++wq) {
-                                const uint2 a = ptx::lds_v2(warp_stat_s + 16u * wq);
-                                const uint2 b = ptx::lds_v2(warp_stat_s + 16u * wq + 8u);
-                                tau_min = fminf(tau_min, (int)a.x == ic ? __uint_as_float(a.y) : -CUDART_INF_F);
-                                ratio_min = fminf(ratio_min, (int)b.x == ic ? __uint_as_float(b.y) : -CUDART_INF_F);
-                            }
-                            if (!(bound < tau_min || k_max < ratio_min)) dead &= ~(1u << qt);
-                            rest_dead = rest_dead && k_max_rest < ratio_min;  // this key tile and every later one of the graph
-                        }
+                    for (int u = 0; u < U; ++u) {
+                        dead[u] = (1u << NQT) - 1u;
+                        bool rest = false;
+                        if (u * 32 + lane < nbatch) dead[u] = evaluate(j0 + u * 32 + lane, rest);
+                        seg_done = seg_done || __any_sync(FULL, rest);
                     }
-                    const unsigned skip_mask = __ballot_sync(FULL, dead == (1u << NQT) - 1u);
-                    const bool seg_done = __any_sync(FULL, rest_dead);
-                    const int nb = min(32, seg_hi - j0);
-                    for (int l = 0; l < nb; ++l) {
-                        const unsigned dead_l = __shfl_sync(FULL, dead, l);
-                        if (lane != 0 || ((skip_mask >> l) & 1u) || !ok) continue;
-                        const int s = kt % S;
-                        if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit))) continue;
-                        const int key0 = it.key_lo + (j0 + l) * BN;
-                        sStageKey[s] = key0;
-                        sStageDead[s] = (int)dead_l;
-                        n_pairs_live += nq - __popc(dead_l & ((1u << nq) - 1u));
-                        ptx::mbar_arrive_expect_tx(bars.k_full(s), Sh::TILE_BYTES);
-                        for (int ch = 0; ch < Sh::KCH; ++ch)
-                            ptx::tma_load_2d(ptx::smem_u32(sK + s * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmK,
-                                             ch * 64, h * dump_ld + key0, bars.k_full(s));
-                        ++kt;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (u * 32 >= nbatch) break;
+                        const unsigned skip_mask = __ballot_sync(FULL, dead[u] == (1u << NQT) - 1u);
+                        const int nb = min(32, nbatch - u * 32);
+                        for (int l = 0; l < nb; ++l) {
+                            const unsigned dead_l = __shfl_sync(FULL, dead[u], l);
+                            if (lane != 0 || ((skip_mask >> l) & 1u) || !ok) continue;
+                            const int s = kt % S;
+                            if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.k_empty(s), ((kt / S) & 1) ^ 1, sAbort, sb, 2, wait_limit))) continue;
+                            const int key0 = it.key_lo + (j0 + u * 32 + l) * BN;
+                            sStageKey[s] = key0;
+                            sStageDead[s] = (int)dead_l;
+                            n_pairs_live += nq - __popc(dead_l & ((1u << nq) - 1u));
+                            ptx::mbar_arrive_expect_tx(bars.k_full(s), Sh::TILE_BYTES);
+                            for (int ch = 0; ch < Sh::KCH; ++ch)
+                                ptx::tma_load_2d(ptx::smem_u32(sK + s * Sh::TILE_BYTES + ch * Sh::CH_BYTES), &tmK,
+                                                 ch * 64, h * dump_ld + key0, bars.k_full(s));
+                            ++kt;
+                        }
                     }
                     ok = __shfl_sync(FULL, (int)ok, 0) != 0;
                     kt = __shfl_sync(FULL, kt, 0);
-                    if (seg_done) break;  // the lanes after the first dead one were skipped by the same test
+                    if (seg_done) break;  // every tile after the first dead one was skipped by the same test
+                    j0 += nbatch;
                 }
             }
             if (!ok) break;

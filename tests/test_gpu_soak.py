@@ -106,3 +106,60 @@ def test_random_small_shapes_against_the_oracle():
             pu.check_backward(w, fb, pu.run_backward(w, fb, dev))
         finally:
             kb.lib().kmip_debug_fp32_path(0)
+
+
+def _pruned_case(rng, case, seed):
+    """One random batch in the pruned mode: large graphs (sorted keys, skipped tiles) next to small ones,
+    clustered, heavy-tailed or unstructured values; sampled rows against a dense recomputation."""
+    H = int(rng.integers(1, 4))
+    d = int(rng.choice([16, 32, 64, 128]))
+    k = int(rng.choice([1, 8, 16, 32, 33, 64, 100]))
+    if d == 128 and k > 64:
+        k = 64
+    sizes = [int(rng.integers(8192, 30000)) for _ in range(int(rng.integers(1, 3)))]
+    sizes += [int(rng.integers(0, 9000)) for _ in range(int(rng.integers(0, 6)))]
+    while sum(sizes) < 32768:
+        sizes.append(int(rng.integers(2000, 12000)))
+    order = rng.permutation(len(sizes))
+    sizes = [sizes[i] for i in order]
+    N = sum(sizes)
+    kind = int(rng.integers(0, 3))
+    torch.manual_seed(seed * 100003 + case)
+    if kind == 1:    # clusters shared by Q and K
+        C = int(rng.choice([8, 32, 64]))
+        lab = torch.randint(0, C, (N,), device="cuda")
+        cen = torch.randn(C, H, d, device="cuda")
+        Q = cen[lab] + 0.2 * torch.randn(N, H, d, device="cuda")
+        K = cen[lab] + 0.2 * torch.randn(N, H, d, device="cuda")
+    else:
+        Q, K = torch.randn(N, H, d, device="cuda"), torch.randn(N, H, d, device="cuda")
+        if kind == 2:  # a few heavy keys
+            K[torch.rand(N, device="cuda") < 0.01] *= 5.0
+    Q, K = Q.bfloat16(), K.bfloat16()
+    V = torch.randn(N, H, d, device="cuda").bfloat16()
+    offs = torch.tensor(np.concatenate([[0], np.cumsum(sizes)]), dtype=torch.int32, device="cuda")
+    what = f"case {case} seed {seed}: sizes={sizes} H={H} d={d} k={k} kind={kind}"
+    for _ in range(2):
+        fb = kb.forward(Q, K, V, offs, k, kb.KMIP_BF16_TC_PRUNED)   # raises on a device-side status
+        idx, sc = fb.topk_idx, fb.topk_score
+        lo, hi = offs[:-1].long(), offs[1:].long()
+        g = torch.searchsorted(hi.contiguous(), torch.arange(N, device="cuda"), right=True)
+        lo_r, hi_r = lo[g][:, None, None], hi[g][:, None, None]
+        valid = torch.arange(k, device="cuda")[None, None, :] < torch.clamp(hi_r - lo_r, max=k)
+        assert bool((((idx >= lo_r) & (idx < hi_r)) | ~valid).all()), what + ": index outside the query's graph"
+        assert bool(((idx == -1) | valid).all()) and bool(((idx >= 0) | ~valid).all()), what + ": wrong padding"
+        for r in torch.randint(0, N, (48,), device="cuda").tolist():
+            a, b = int(lo[g[r]]), int(hi[g[r]])
+            s = (Q[r].float()[:, None, :] * K[a:b].float().permute(1, 0, 2)).sum(-1)   # [H, n]
+            kk = min(k, b - a)
+            best = torch.topk(s, kk, dim=1).values
+            assert torch.allclose(sc[r, :, :kk], best, rtol=2e-4, atol=2e-4), what + f": row {r} lost a key"
+            got = torch.gather(s, 1, (idx[r, :, :kk].long() - a))
+            assert torch.allclose(got, sc[r, :, :kk], rtol=2e-4, atol=2e-4), what + f": row {r} index and score disagree"
+
+
+@pytest.mark.parametrize("seed,cases", [(21, 60)])
+def test_random_shapes_pruned_mode(seed, cases):
+    rng = np.random.default_rng(seed)
+    for case in range(cases):
+        _pruned_case(rng, case, seed)
