@@ -46,6 +46,13 @@ def test_workspace_bytes_host_only(kb):
     small = kb.kmip_attn_workspace_bytes(20_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
     assert 20_000 * 4 * 32 * 2 < small < 20_000 * 4 * 32 * 2 + (1 << 20)    # small problems keep their row order: K copy only
     assert 256 < kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_FP32_EXACT, kb.PASS_FORWARD) < (1 << 20)
+    # pruned mode: 16 bytes per node + 4 per (node, head) + (d + 4) floats per (128 nodes, head) for the key tiles
+    # and three times that for the query tiles of the work items; the same as the plain mode below 32768 nodes
+    fp = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_FORWARD)
+    extra = 500_000 * (16 + 4 * 4) + 4 * (500_000 // 128 + 3) * 4 * 36 * 4
+    assert f + 500_000 * 16 < fp < f + extra + (1 << 16)
+    assert kb.kmip_attn_workspace_bytes(20_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_FORWARD) == small
+    assert kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_BACKWARD) == b
     pairs = 500_000 * 4 * 32
     assert 24 * pairs < b < 26 * pairs          # p, dS, 16-byte hit records: 24 bytes per selected pair + O(N*H)
     for bad in [dict(d=24), dict(k=129), dict(mode=7)]:

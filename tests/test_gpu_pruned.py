@@ -110,3 +110,30 @@ def test_workspace_of_the_pruned_mode_is_reported_and_enforced():
     fb = kb.ForwardBuffers(N, 1, H, d, k, w.mode)
     small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
     assert kb.kmip_attn_forward(Q, K, V, offs, k, w.mode, fb.out, fb.topk_idx, fb.topk_score, small) == kb.KMIP_ERR_WORKSPACE
+
+
+def test_layer_with_pruning_matches_layer_without():
+    """The layer's prune option only changes the mode of the attention core."""
+    from paper_2604_03815_b200.layer import KMIPSelfAttention
+
+    torch.manual_seed(5)
+    N, d_model = 33000, 64
+    cen = torch.randn(16, d_model, device="cuda")
+    x = (cen[torch.randint(0, 16, (N,), device="cuda")] + 0.2 * torch.randn(N, d_model, device="cuda")).bfloat16()
+    a = KMIPSelfAttention(d_model, 2, 32, 16)
+    b = KMIPSelfAttention(d_model, 2, 32, 16, prune=True)
+    b.load_state_dict(a.state_dict())
+    assert b.mode == kb.KMIP_BF16_TC_PRUNED
+    xa, xb = x.clone().requires_grad_(True), x.clone().requires_grad_(True)
+    ya, ia = a(xa, return_indices=True)
+    yb, ib = b(xb, return_indices=True)
+    assert float((ia == ib).float().mean()) > 0.999
+    same = (ia == ib).all(dim=-1).all(dim=-1)
+    assert torch.allclose(ya[same].float(), yb[same].float(), rtol=2e-2, atol=2e-2)
+    ya.float().square().sum().backward()
+    yb.float().square().sum().backward()
+    assert torch.isfinite(xb.grad.float()).all()
+    rel = (xa.grad.float() - xb.grad.float()).norm() / xa.grad.float().norm()
+    assert float(rel) < 2e-2
+    b.set_k(8)
+    assert b(x).shape == (N, d_model)
