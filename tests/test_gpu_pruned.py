@@ -137,3 +137,55 @@ def test_layer_with_pruning_matches_layer_without():
     assert float(rel) < 2e-2
     b.set_k(8)
     assert b(x).shape == (N, d_model)
+
+
+def _dense_check(Q, K, V, offs, k, n_rows=64, seed=0):
+    """Sampled rows of a pruned-mode forward against dense fp32 scores computed by torch on the GPU:
+    the kept scores are the row's k largest and every index scores what the list says."""
+    fb = kb.forward(Q, K, V, offs, k, kb.KMIP_BF16_TC_PRUNED)   # raises on a device-side status
+    N = Q.shape[0]
+    lo, hi = offs[:-1].long(), offs[1:].long()
+    g = torch.searchsorted(hi.contiguous(), torch.arange(N, device="cuda"), right=True)
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    for r in torch.randint(0, N, (n_rows,), device="cuda", generator=gen).tolist():
+        a, b = int(lo[g[r]]), int(hi[g[r]])
+        s = (Q[r].float()[:, None, :] * K[a:b].float().permute(1, 0, 2)).sum(-1)   # [H, n]
+        kk = min(k, b - a)
+        best = torch.topk(s, kk, dim=1).values
+        tol = 2e-4 * max(1.0, float(best.abs().max()))
+        assert float((fb.topk_score[r, :, :kk] - best).abs().max()) <= tol, f"row {r}: kept scores are not the k largest"
+        idx = fb.topk_idx[r, :, :kk].long()
+        assert bool(((idx >= a) & (idx < b)).all())
+        got = torch.gather(s, 1, idx - a)
+        assert float((got - fb.topk_score[r, :, :kk]).abs().max()) <= tol, f"row {r}: index and score disagree"
+        assert all(len(set(row)) == kk for row in idx.tolist()), f"row {r}: a key is listed twice"
+    return fb
+
+
+@pytest.mark.parametrize("case", ["zero_keys", "identical_keys", "negative_scores", "one_giant_key", "zero_queries",
+                                  "two_scales"])
+def test_degenerate_values(case):
+    """Values that stress the bounds: thresholds that stay at or below zero (the norm bound must not fire),
+    radii of zero, norms spread over many orders of magnitude."""
+    torch.manual_seed(3)
+    N, H, d, k = 34000, 2, 32, 16
+    offs = torch.tensor([0, 9000, 9100, N], dtype=torch.int32, device="cuda")
+    Q, K = torch.randn(N, H, d, device="cuda"), torch.randn(N, H, d, device="cuda")
+    if case == "zero_keys":
+        K.zero_()
+    elif case == "identical_keys":
+        K[:] = K[0]
+    elif case == "negative_scores":
+        base = torch.randn(H, d, device="cuda")
+        Q = base + 0.1 * torch.randn(N, H, d, device="cuda")
+        K = -base + 0.1 * torch.randn(N, H, d, device="cuda")
+    elif case == "one_giant_key":
+        K[12345] *= 1.0e4
+    elif case == "zero_queries":
+        Q[::3] = 0.0
+    elif case == "two_scales":
+        K[: N // 2] *= 1.0e-3
+        Q[N // 2:] *= 1.0e3
+    V = torch.randn(N, H, d, device="cuda")
+    fb = _dense_check(Q.bfloat16(), K.bfloat16(), V.bfloat16(), offs, k)
+    assert torch.isfinite(fb.out.float()).all()
