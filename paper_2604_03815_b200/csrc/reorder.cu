@@ -112,6 +112,85 @@ graph_sort_kernel(const int32_t* __restrict__ offs, int G, int N, const unsigned
     }
 }
 
+// The same sort, but stable (rows of a bucket stay in row order), so that the order - and with it which of
+// several keys with exactly equal scores the pruned sweep meets first - does not depend on the timing of
+// atomics.  Each of the 32 warps owns a contiguous chunk of the graph's rows and a histogram row of its
+// own in shared memory; after the counts are turned into start positions per (warp, bucket), a warp places
+// its rows 32 at a time, ranking equal codes inside the 32 with a match vote.  32 * 2^BITS counters:
+// BITS <= 10.
+template <int BITS>
+__global__ void __launch_bounds__(kSortThreads)
+graph_sort_stable_kernel(const int32_t* __restrict__ offs, int G, int N, const unsigned short* __restrict__ code,
+                         int* __restrict__ perm, const StatusBlock* __restrict__ sb) {
+    if (sb->status != KMIP_OK) return;
+    constexpr int kBuckets = 1 << BITS;
+    constexpr int kWarpsS = kSortThreads / 32;
+    static_assert(kBuckets <= kSortThreads, "one thread per bucket in the scan");
+    extern __shared__ int s_hist[];  // [kWarpsS][kBuckets]
+    __shared__ int s_warp[32];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int n_graphs = offs ? G : 1;
+    for (int g = blockIdx.x; g < n_graphs; g += gridDim.x) {
+        const int lo = offs ? __ldg(offs + g) : 0, hi = offs ? __ldg(offs + g + 1) : N;
+        if (hi - lo < kMinRowsToSort) {
+            for (int r = lo + tid; r < hi; r += kSortThreads) perm[r] = r;
+            continue;
+        }
+        __syncthreads();
+        for (int x = tid; x < kWarpsS * kBuckets; x += kSortThreads) s_hist[x] = 0;
+        __syncthreads();
+        const int chunk = (hi - lo + kWarpsS - 1) / kWarpsS;
+        const int c_lo = min(hi, lo + wid * chunk), c_hi = min(hi, c_lo + chunk);
+        int* mine = s_hist + wid * kBuckets;
+        for (int r = c_lo + lane; r < c_hi; r += 32) atomicAdd(&mine[code[r]], 1);  // contention inside the warp only
+        __syncthreads();
+        // thread b < kBuckets: total of bucket b, exclusive scan over buckets, then start of every warp's share
+        int total = 0;
+        if (tid < kBuckets)
+            for (int w = 0; w < kWarpsS; ++w) total += s_hist[w * kBuckets + tid];
+        int incl = total;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_warp[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            int v = s_warp[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, v, o);
+                if (lane >= o) v += t;
+            }
+            s_warp[lane] = v;
+        }
+        __syncthreads();
+        if (tid < kBuckets) {
+            int start = lo + (wid ? s_warp[wid - 1] : 0) + incl - total;
+            for (int w = 0; w < kWarpsS; ++w) {
+                const int c = s_hist[w * kBuckets + tid];
+                s_hist[w * kBuckets + tid] = start;
+                start += c;
+            }
+        }
+        __syncthreads();
+        for (int r0 = c_lo; r0 < c_hi; r0 += 32) {
+            const int r = r0 + lane;
+            const bool live = r < c_hi;
+            const unsigned cd = live ? code[r] : 0xFFFFFFFFu;  // idle lanes match among themselves only
+            const unsigned same = __match_any_sync(0xFFFFFFFFu, cd);
+            if (live) {
+                const int rank = __popc(same & ((1u << lane) - 1u));
+                perm[mine[cd] + rank] = r;
+            }
+            __syncwarp();
+            if (live && (same >> lane) == 1u) mine[cd] += __popc(same);  // the group's highest lane moves the cursor
+            __syncwarp();
+        }
+    }
+}
+
 // Qp[p, :] = Q[perm[p], :], 16 bytes per thread.
 __global__ void gather_rows_kernel(const uint4* __restrict__ Q, const int* __restrict__ perm, uint4* __restrict__ Qp,
                                    long long n_vec, int vec_per_row, const StatusBlock* __restrict__ sb) {
@@ -298,7 +377,7 @@ cudaError_t launch_reorder_queries(const FwdArgs& a, const FwdWorkspace& w) {
         kern<<<w.max_items, kAssignThreads, smem, a.stream>>>(
             static_cast<const __nv_bfloat16*>(a.Q), static_cast<const __nv_bfloat16*>(a.K), HD,
             reinterpret_cast<const WorkItem*>(a.ws + w.items_off), sb, a.graph_offsets, a.G, nullptr, nullptr, code);
-        graph_sort_kernel<kPivotBits><<<std::min(n_graphs, 148 * 2), kSortThreads, (1 << kPivotBits) * 4, a.stream>>>(
+        graph_sort_stable_kernel<kPivotBits><<<std::min(n_graphs, 148 * 2), kSortThreads, (32 << kPivotBits) * 4, a.stream>>>(
             a.graph_offsets, a.G, (int)a.N, code, perm, sb);
     } else {
         query_code_kernel<<<(unsigned)((a.N * 32 + 255) / 256), 256, 0, a.stream>>>(
@@ -338,8 +417,11 @@ cudaError_t launch_reorder_keys(const FwdArgs& a, const FwdWorkspace& w) {
     if (err != cudaSuccess) return err;
     kern<<<w.max_items, kAssignThreads, smem, a.stream>>>(K, K, HD, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), sb,
                                                           a.graph_offsets, a.G, norm2, gmax, code);
-    graph_sort_kernel<kKeyCodeBits2><<<std::min(n_graphs, 148 * 2), kSortThreads, (1 << kKeyCodeBits2) * 4, a.stream>>>(
-        a.graph_offsets, a.G, (int)a.N, code, kperm, sb);
+    auto sort = graph_sort_stable_kernel<kKeyCodeBits2>;
+    constexpr int sort_smem = (32 << kKeyCodeBits2) * 4;
+    err = cudaFuncSetAttribute(sort, cudaFuncAttributeMaxDynamicSharedMemorySize, sort_smem);
+    if (err != cudaSuccess) return err;
+    sort<<<std::min(n_graphs, 148 * 2), kSortThreads, sort_smem, a.stream>>>(a.graph_offsets, a.G, (int)a.N, code, kperm, sb);
     const int vec_per_row = a.d * 2 / 16;
     const long long n_vec = (long long)a.N * a.H * vec_per_row;
     pack_keys_perm_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, a.stream>>>(

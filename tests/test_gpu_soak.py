@@ -58,19 +58,22 @@ def test_random_shapes(seed, force_wide, cases):
         _one_case(rng, case, seed, force_wide)
 
 
-@pytest.mark.parametrize("cfg,kw", [(3, {}), (4, {"N": 100000, "d": 128, "H": 1}), (4, {"N": 120000, "k": 64})])
-def test_large_runs_are_bit_identical(cfg, kw):
+@pytest.mark.parametrize("cfg,kw,pruned", [(3, {}, False), (4, {"N": 100000, "d": 128, "H": 1}, False),
+                                           (4, {"N": 120000, "k": 64}, False), (4, {"N": 120000}, True),
+                                           (5, {"n_per_graph": 30000}, True)])
+def test_large_runs_are_bit_identical(cfg, kw, pruned):
     """The selection is exact whatever the timing of the pipeline, so repeated runs on the same
     inputs must agree bit for bit; a run that read an accumulator or a key stage at the wrong
     moment would not."""
     w = wl.make_config(cfg, **kw)
-    dt = kb.storage_dtype(w.mode)
+    mode = kb.KMIP_BF16_TC_PRUNED if pruned else w.mode  # the pruned mode's key and row orders come from stable sorts
+    dt = kb.storage_dtype(mode)
     Q, K, V = (torch.from_numpy(getattr(w, n)).to("cuda", dt) for n in "QKV")
     offs = torch.from_numpy(w.graph_offsets).cuda()
-    fb = kb.ForwardBuffers(w.N, len(w.graph_offsets) - 1, w.H, w.d, w.k, w.mode)
+    fb = kb.ForwardBuffers(w.N, len(w.graph_offsets) - 1, w.H, w.d, w.k, mode)
     ref = None
     for _ in range(6):
-        assert kb.kmip_attn_forward(Q, K, V, offs, w.k, w.mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace) == kb.KMIP_OK
+        assert kb.kmip_attn_forward(Q, K, V, offs, w.k, mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace) == kb.KMIP_OK
         torch.cuda.synchronize()
         assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK
         cur = (fb.topk_idx.clone(), fb.topk_score.clone(), fb.out.clone())
