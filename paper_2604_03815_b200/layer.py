@@ -57,7 +57,10 @@ class KMIPSelfAttention(torch.nn.Module):
     """x [N, d_model] -> [N, d_model]: per head h, Q^h = x W_Q^h, K^h = x W_K^h, V^h = x W_V^h,
     O^h = kMIP-Attn(Q^h, K^h, V^h) restricted to each graph, y = sum_h O^h W_O^h (Eq. 2).
 
-    d_head must be 16, 32, 64 or 128 and k <= 128.  dtype bfloat16 selects the tensor-core mode,
+    k <= 128.  The kernels take head widths 16, 32, 64 and 128; any other d_head <= 128 (the paper's own
+    study uses 10) is zero-padded to the next of those behind the projections, which leaves every inner
+    product unchanged, with the queries scaled by sqrt(padded / d_head) so that the softmax still divides
+    the scores by sqrt(d_head) as Eq. 1 does.  dtype bfloat16 selects the tensor-core mode,
     float32 the fp32 mode.  attn_dropout is the dropout rate on the k attention weights, active in
     training mode only (the paper's graph models use 0.5); every forward call draws a fresh seed
     from torch's CPU generator, so torch.manual_seed makes a run repeatable.  prune=True selects the
@@ -70,6 +73,9 @@ class KMIPSelfAttention(torch.nn.Module):
         if dtype not in (torch.bfloat16, torch.float32):
             raise ValueError("dtype must be torch.bfloat16 or torch.float32")
         self.d_model, self.H, self.d, self.k = d_model, num_heads, d_head, k
+        if not 1 <= d_head <= 128:
+            raise ValueError("d_head must be in 1..128")
+        self.d_pad = next(w for w in (16, 32, 64, 128) if w >= d_head)
         if not 0.0 <= attn_dropout < 1.0:
             raise ValueError("attn_dropout must be in [0, 1)")
         self.attn_dropout = float(attn_dropout)
@@ -94,8 +100,12 @@ class KMIPSelfAttention(torch.nn.Module):
         q = self.w_q(x).view(N, self.H, self.d)
         k = self.w_k(x).view(N, self.H, self.d)
         v = self.w_v(x).view(N, self.H, self.d)
+        if self.d_pad != self.d:
+            pad = (0, self.d_pad - self.d)
+            q = torch.nn.functional.pad(q * math.sqrt(self.d_pad / self.d), pad)
+            k, v = torch.nn.functional.pad(k, pad), torch.nn.functional.pad(v, pad)
         drop = self.attn_dropout if self.training else 0.0
         seed = int(torch.randint(0, 2 ** 62, (1,)).item()) if drop > 0.0 else 0
         o, idx = KMIPAttentionFunction.apply(q, k, v, graph_offsets, self.k, self.mode, drop, seed)
-        y = self.w_o(o.reshape(N, self.H * self.d))
+        y = self.w_o(o[..., :self.d].reshape(N, self.H * self.d))
         return (y, idx) if return_indices else y

@@ -31,7 +31,8 @@ def _reference(x, wq, wk, wv, wo, idx, H, d, rounding):
     return r(o.reshape(N, H * d) @ wo.T), q, k
 
 
-@pytest.mark.parametrize("dtype,d_head,k", [(torch.bfloat16, 16, 8), (torch.bfloat16, 32, 16), (torch.float32, 32, 5)])
+@pytest.mark.parametrize("dtype,d_head,k", [(torch.bfloat16, 16, 8), (torch.bfloat16, 32, 16), (torch.float32, 32, 5),
+                                            (torch.float32, 10, 10), (torch.bfloat16, 40, 6)])
 def test_layer_forward_and_gradients(dtype, d_head, k):
     from paper_2604_03815_b200.layer import KMIPSelfAttention
 
