@@ -346,6 +346,26 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
     const int n_items = sb->n_items;
     const long long total = (long long)n_items * H;
+    // Tail of the persistent schedule.  A unit of work is a (work item, head) pair and takes the same time
+    // whether one or all of its query tiles hold rows (the warp groups run side by side), so when the units
+    // do not divide by the grid, the last `left` ones would keep a few CTAs busy for a whole unit while the
+    // rest idle.  Those units are cut into their 128-row query tiles instead, one CTA each - a CTA with a
+    // single busy warp group gets through its key tiles faster - provided the pieces fit one wave.
+    long long n_whole = total, n_units = total;
+    if (!PRUNE && !DUMP && NQT > 1 && total > (long long)gridDim.x) {
+        const long long left = total % gridDim.x;
+        if (left * NQT <= (long long)gridDim.x) { n_whole = total - left; n_units = n_whole + left * NQT; }
+    }
+    // unit number -> head and work item (all roles decode it the same way); false: a piece without rows
+    auto unit = [&](long long w, int& h, WorkItem& it) -> bool {
+        long long base = w;
+        int piece = -1;
+        if (w >= n_whole) { base = n_whole + (w - n_whole) / NQT; piece = (int)((w - n_whole) % NQT); }
+        h = (int)(base / n_items);
+        it = items[base % n_items];
+        if (piece >= 0) { it.row0 += piece * BM; it.nrows = min(BM, it.nrows - piece * BM); }
+        return it.nrows > 0;
+    };
 
     if (PRUNE && warp == NEPI) {
         // ------------------------------------------------------------------ TMA producer, pruned sweep
@@ -503,9 +523,10 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (lane == 0) {
             int kt = 0, ic = 0;
             bool ok = true;
-            for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const int h = (int)(w / n_items);
-                const WorkItem it = items[w % n_items];
+            for (long long w = blockIdx.x; ok && w < n_units; w += gridDim.x) {
+                int h;
+                WorkItem it;
+                if (!unit(w, h, it)) continue;
                 if (!(ok = wait_or_abort<kRelaxedPollNs>(bars.q_empty(), (ic & 1) ^ 1, sAbort, sb, 1, wait_limit))) break;
                 ptx::mbar_arrive_expect_tx(bars.q_full(), NQT * Sh::TILE_BYTES);
                 for (int qt = 0; qt < NQT; ++qt)
@@ -560,8 +581,10 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             int kt = 0, ic = 0;
             bool ok = true;
             long long w_kfull = 0, w_tempty = 0, t_begin = clock64();
-            for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const WorkItem it = items[w % n_items];
+            for (long long w = blockIdx.x; ok && w < n_units; w += gridDim.x) {
+                int h_unused;
+                WorkItem it;
+                if (!unit(w, h_unused, it)) continue;
                 const int nq = (it.nrows + BM - 1) / BM;  // query tiles of the item that hold rows
                 if (!(ok = wait_or_abort<0>(bars.q_full(), ic & 1, sAbort, sb, 3, wait_limit))) break;
                 ptx::tc_fence_after();
@@ -647,9 +670,10 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         bool ok = true;
         long long w_tfull = 0, t_work = 0, t_begin = clock64();
         long long prof[4] = {0, 0, 0, 0};
-        for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
-            const int h = (int)(w / n_items);
-            const WorkItem it = items[w % n_items];
+        for (long long w = blockIdx.x; ok && w < n_units; w += gridDim.x) {
+            int h;
+            WorkItem it;
+            if (!unit(w, h, it)) continue;
             const bool active = qt * BM < it.nrows;  // an inactive query tile only keeps the barriers in step
             const int local = qt * BM + quarter * 32 + lane;
             const bool rvalid = local < it.nrows;
