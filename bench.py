@@ -297,25 +297,22 @@ def run_ours(args, w):
                                            fbp.topk_idx, fbp.topk_score, bb.dQ, bb.dK, bb.dV, bb.workspace)
                 assert rc == kb.KMIP_OK, kb.status_string(rc)
 
-        counters = torch.zeros(8 * 256, dtype=torch.int64, device=dev)
-        kb.sweep_counters(counters)
         for _ in range(3):
             step_pruned()
         torch.cuda.synchronize()
-        kb.sweep_counters(None)
         assert kb.kmip_last_status(fbp.workspace) == kb.KMIP_OK
+        cnt = kb.kmip_attn_sweep_counters(fbp.workspace)   # of the last forward call
         kb.kmip_profile_enable(min(args.steps, 256))
         secs_p = timed(step_pruned, args.steps)
         st_p, nf_p, _ = kb.kmip_profile_read()
         kb.kmip_profile_enable(0)
-        cnt = counters.cpu().numpy().reshape(-1, 8)
         _, t_p = kdist.aggregate_throughput(float(w.n_scores) * args.steps, secs_p)
         pruned = {
             "mode": "KMIP_BF16_TC_PRUNED", "ms_per_step": 1e3 * t_p / args.steps,
             "value": float(w.n_scores) * args.steps / t_p, "unit": UNIT,
             "plan_ms": st_p["plan"] / max(1, nf_p), "sweep_ms": st_p["score_select"] / max(1, nf_p),
-            "key_tiles_loaded_frac": float(cnt[:, 1].sum() / max(1, cnt[:, 0].sum())),
-            "pairs_scored_frac": float(cnt[:, 3].sum() / max(1, cnt[:, 2].sum())),
+            "key_tiles_loaded_frac": float(cnt[1] / max(1, cnt[0])),
+            "pairs_scored_frac": float(cnt[3] / max(1, cnt[2])),
             "note": "same results (exact pruning); scores/s counts the scores of the definition, not the ones computed",
         }
         del fbp

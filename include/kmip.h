@@ -16,13 +16,17 @@
  *            graph_offsets : int32 [G+1], offsets[0] = 0, non-decreasing, offsets[G] = N.
  *   memory   every pointer is DEVICE memory owned by the caller, 16-byte aligned, and stays
  *            valid until the work enqueued on `stream` has finished.  The library allocates
- *            no device memory and keeps no state between calls; `workspace` is caller-owned
- *            scratch whose contents are undefined between calls.  Its first 256 bytes are
- *            a status block that kmip_last_status reads.
+ *            no device memory and keeps no state between calls, with two documented exceptions:
+ *            kmip_attn_forward_static_scratch (a built-in scratch array and its cached device
+ *            address) and the kmip_profile_* calls (process-wide CUDA events).  `workspace` is
+ *            caller-owned scratch whose contents are undefined between calls.  Its first 256
+ *            bytes are a status block that kmip_last_status reads.
  *   async    calls validate their arguments on the host, enqueue kernels on `stream`
  *            (a cudaStream_t passed as void*, NULL = default stream) and return without
  *            synchronising.  KMIP_OK means "enqueued".  Problems only the device can see
- *            (malformed offsets, an expired bounded wait) are recorded in the status block.
+ *            (malformed offsets, an expired bounded wait) are recorded in the status block;
+ *            the kernels enqueued after such a problem return without writing, so the call's
+ *            outputs are undefined whenever the status word is not KMIP_OK.
  *   errors   nothing is enqueued when a call returns a status other than KMIP_OK.
  */
 #ifndef KMIP_H_
@@ -87,7 +91,8 @@ int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_
  * A graph with n < k nodes keeps all n and pads: topk_idx = -1, topk_score = -inf, weight 0.
  * graph_offsets may be NULL, meaning one graph [0, N) (G is then ignored).
  * N = 0 returns KMIP_OK and enqueues nothing.
- * Inputs: Q, K, V, graph_offsets.  Outputs (fully overwritten): out, topk_idx, topk_score.
+ * Inputs: Q, K, V, graph_offsets.  Outputs (fully overwritten when the device status word stays
+ * KMIP_OK, undefined otherwise): out, topk_idx, topk_score.
  * In KMIP_BF16_TC mode the selection uses tensor-core scores, so a key whose exact score
  * differs from the k-th best by less than the fp32 accumulation error may swap with it.
  */
@@ -123,7 +128,7 @@ int kmip_attn_backward(const void *Q, const void *K, const void *V,
 
 /*
  * Training variants with attention dropout on the k softmax weights (the paper trains its LRGB and
- * City-Networks models with attention dropout 0.5 and its point-cloud models with 0; App. G).
+ * City-Networks models with attention dropout 0.5 and its point-cloud models with 0; App. H).
  * Each weight p_t of Algorithm 1 line 5 is kept with probability 1 - drop_p and divided by
  * 1 - drop_p, independently per (query, head, slot):
  *   out[i,h,:] = sum_t f_t p_t V[topk_idx_t, h, :],   f_t = 1/(1 - drop_p) or 0.
@@ -151,7 +156,7 @@ int kmip_attn_backward_dropout(const void *Q, const void *K, const void *V,
                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * Diagnostic of the paper's App. H (cumulative attention weight): for every query node and head,
+ * Diagnostic of the paper's App. I (cumulative attention weight): for every query node and head,
  * the share of the FULL softmax over all nodes of its graph that falls on the k keys kept by the
  * forward pass,
  *   mass[i,h] = sum_t exp(topk_score[i,h,t] / sqrt(d)) / sum_j exp(q_i^h . k_j^h / sqrt(d)),
@@ -187,10 +192,11 @@ int kmip_attn_topk_mass(const void *Q, const void *K,
  *     refused with KMIP_ERR_TOO_LARGE before anything is enqueued.  In tensor-core mode the scratch
  *     is dominated by one bf16 copy of K (and one of Q from 32768 nodes on), so the limit is about
  *     N*H*d <= 4.1 million elements (2 million from 32768 nodes on)
- *     (e.g. 32 000 nodes at H = 4, d = 32); fp32 mode needs 16 bytes per 128 nodes and per graph.
+ *     (e.g. 32 000 nodes at H = 4, d = 32); fp32 mode needs 20 bytes per 128 nodes and per graph.
  *   - device_status (DEVICE pointer, may be NULL): if given, the device status word of this call
  *     (KMIP_OK, KMIP_ERR_TIMEOUT or KMIP_ERR_BAD_OFFSETS) is copied there on `stream` after the
- *     kernels, since there is no workspace for kmip_last_status to read.
+ *     kernels, since there is no workspace for kmip_last_status to read (N = 0: KMIP_OK is
+ *     stored there, nothing else is enqueued).
  *   - the call itself calls no cudaMalloc / cudaFree or any other allocating routine.  The first call
  *     on each device looks up the array's device address (cudaGetSymbolAddress, with that device
  *     current) and caches it; make that first call outside any stream capture.
@@ -212,6 +218,16 @@ int kmip_attn_forward_static_scratch(const void *Q, const void *K, const void *V
  * not needed on the hot path.
  */
 int kmip_last_status(const void *workspace, void *stream, int *device_status);
+
+/*
+ * Work counters of the pruned sweep (KMIP_BF16_TC_PRUNED; the paper has no counterpart).  Synchronises
+ * `stream`, then reads from the status block of `workspace` (the forward workspace of the last
+ * call) counters[4] = {key tiles of all work items, key tiles loaded (one end marker per work item
+ * included), (key tile, query tile) pairs, pairs scored}, summed over the sweep's CTAs.  All zero
+ * after a call in another mode.  counters: HOST memory, four int64.  Returns KMIP_ERR_CUDA if the
+ * synchronisation or the copy fails.
+ */
+int kmip_attn_sweep_counters(const void *workspace, void *stream, int64_t *counters);
 
 /*
  * Optional per-stage timing for benchmarks; the paper has no counterpart (its Fig. 3 reports a

@@ -204,7 +204,7 @@ int kmip_oracle_forward_rows(const float *Q, const float *K, const float *V,
 }
 
 /*
- * Diagnostic of the paper's App. H ("cumulative attention weight"): how much of the FULL softmax
+ * Diagnostic of the paper's App. I ("cumulative attention weight"): how much of the FULL softmax
  * over all keys of the query's graph falls on the k keys with the largest scores,
  *   mass[i,h] = sum_{t<k} softmax_j(q_i.k_j / sqrt(d))_(t)     (1 when the graph has <= k nodes).
  * Plain definition: every score of the row, a stable log-sum-exp over all of them, and the sum of
@@ -265,7 +265,7 @@ int kmip_oracle_topk_mass(const float *Q, const float *K, const int32_t *graph_o
 
 /*
  * Attention dropout on the k softmax weights (the paper trains with it: 0.5 on the LRGB and
- * City-Networks models, 0.0 on point clouds; App. G): each weight is kept with probability
+ * City-Networks models, 0.0 on point clouds; App. H): each weight is kept with probability
  * 1 - drop and divided by 1 - drop ("inverted" dropout), independently per (query, head, slot).
  * The draw for slot t of query i, head h is a counter-based uniform: the splitmix64 finaliser
  * of seed + (pair + 1) * 0x9E3779B97F4A7C15 with pair = (i*H + h)*k + t, top 24 bits / 2^24;

@@ -29,6 +29,12 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libkmip.so"
 _lib = None
 
 
+class TestOptions(ctypes.Structure):
+    """kmip_test_options_t of include/kmip_test.h."""
+    _fields_ = [("wait_limit_cycles", ctypes.c_int64), ("drop_first_tile", ctypes.c_int32),
+                ("fp32_path", ctypes.c_int32)]
+
+
 class KmipError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -71,8 +77,16 @@ def lib() -> ctypes.CDLL:
         L.kmip_profile_enable.argtypes = [ctypes.c_int]
         L.kmip_profile_read.restype = ctypes.c_int
         L.kmip_profile_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
-        L.kmip_debug_tc_scores.restype = ctypes.c_int
-        L.kmip_debug_tc_scores.argtypes = [P, P, i64, i32, i32, P, P, sz, P]
+        L.kmip_attn_sweep_counters.restype = ctypes.c_int
+        L.kmip_attn_sweep_counters.argtypes = [P, P, ctypes.POINTER(ctypes.c_int64)]
+        # kmip_test.h
+        L.kmip_test_tc_scores.restype = ctypes.c_int
+        L.kmip_test_tc_scores.argtypes = [P, P, i64, i32, i32, P, P, sz, P]
+        L.kmip_test_sweep_order.restype = ctypes.c_int
+        L.kmip_test_sweep_order.argtypes = [P, i64, i32, i32, i32, i32, ctypes.c_int, P, ctypes.POINTER(i32), P]
+        L.kmip_test_attn_forward.restype = ctypes.c_int
+        L.kmip_test_attn_forward.argtypes = [P, P, P, P, i32, i64, i32, i32, i32, ctypes.c_int, P, P, P, P, sz, P,
+                                             ctypes.POINTER(TestOptions)]
         _lib = L
     return _lib
 
@@ -199,25 +213,51 @@ def kmip_profile_read():
     return dict(zip(STAGES, list(ms))), int(calls[0]), int(calls[1])
 
 
-def kmip_debug_tc_scores(Q, K, scores, workspace, stream=None) -> int:
-    """Test hook: dense q.k scores [H, N, N] of one small graph through the tensor-core pipeline."""
+def kmip_test_tc_scores(Q, K, scores, workspace, stream=None) -> int:
+    """kmip_test.h: dense q.k scores [H, N, N] of one small graph through the tensor-core pipeline."""
     N, H, d = Q.shape
-    return int(lib().kmip_debug_tc_scores(_ptr(Q), _ptr(K), N, H, d, _ptr(scores), _ptr(workspace),
-                                          workspace.numel() * workspace.element_size(), _stream(stream)))
+    return int(lib().kmip_test_tc_scores(_ptr(Q), _ptr(K), N, H, d, _ptr(scores), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def kmip_test_attn_forward(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score, workspace, stream=None,
+                           wait_limit_cycles=0, drop_first_tile=0, fp32_path=0) -> int:
+    """kmip_test.h: the forward pass with per-call test options; returns the library's status code."""
+    N, H, d = Q.shape
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    opt = TestOptions(int(wait_limit_cycles), int(drop_first_tile), int(fp32_path))
+    return int(lib().kmip_test_attn_forward(_ptr(Q), _ptr(K), _ptr(V), _ptr(graph_offsets), G, N, H, d, k, mode,
+                                            _ptr(out), _ptr(topk_idx), _ptr(topk_score), _ptr(workspace),
+                                            0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                            _stream(stream), ctypes.byref(opt)))
+
+
+def kmip_test_sweep_order(workspace, N, G, H, d, k, mode, stream=None):
+    """kmip_test.h: (order, rows_per_item) of the last forward call on `workspace`; order[s] is the row the
+    sweep handled at position s (numpy int32 [N])."""
+    import numpy as np
+    order = np.empty(N, dtype=np.int32)
+    rpi = ctypes.c_int32(0)
+    rc = lib().kmip_test_sweep_order(_ptr(workspace), N, G, H, d, k, mode, order.ctypes.data_as(ctypes.c_void_p),
+                                     ctypes.byref(rpi), _stream(stream))
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_test_sweep_order")
+    return order, int(rpi.value)
+
+
+def kmip_attn_sweep_counters(workspace, stream=None):
+    """Work counters of the pruned sweep's last call on `workspace` (synchronises the stream):
+    (key tiles, key tiles loaded, (key tile, query tile) pairs, pairs scored)."""
+    c = (ctypes.c_int64 * 4)()
+    rc = lib().kmip_attn_sweep_counters(_ptr(workspace), _stream(stream), c)
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_attn_sweep_counters")
+    return tuple(int(x) for x in c)
 
 
 # ------------------------------------------------------------------------------------------------
 # Buffer helpers (allocation only)
 # ------------------------------------------------------------------------------------------------
-def sweep_counters(buf) -> None:
-    """Diagnostic hook (not in kmip.h): int64 device tensor of 8 * SMs entries that the pruned sweep fills
-    per CTA with {key tiles, tiles loaded, (key tile, query tile) pairs, pairs scored}; None switches it off."""
-    f = lib().kmip_debug_set_timing
-    f.argtypes = [ctypes.c_void_p]
-    f.restype = None
-    f(ctypes.c_void_p(buf.data_ptr()) if buf is not None else ctypes.c_void_p(0))
-
-
 def storage_dtype(mode: int):
     return torch.float32 if mode == KMIP_FP32_EXACT else torch.bfloat16
 
@@ -246,12 +286,18 @@ class BackwardBuffers:
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
 
 
-def forward(Q, K, V, graph_offsets, k, mode, buffers: ForwardBuffers | None = None, stream=None, check=True):
-    """Allocate (unless given) and run the forward pass; returns the buffers."""
+def forward(Q, K, V, graph_offsets, k, mode, buffers: ForwardBuffers | None = None, stream=None, check=True,
+            fp32_path=0):
+    """Allocate (unless given) and run the forward pass; returns the buffers.  fp32_path != 0 goes through
+    kmip_test_attn_forward to pin which fp32-mode sweep runs (tests only)."""
     N, H, d = Q.shape
     G = 1 if graph_offsets is None else int(graph_offsets.numel()) - 1
     b = buffers or ForwardBuffers(N, G, H, d, k, mode, Q.device)
-    rc = kmip_attn_forward(Q, K, V, graph_offsets, k, mode, b.out, b.topk_idx, b.topk_score, b.workspace, stream)
+    if fp32_path:
+        rc = kmip_test_attn_forward(Q, K, V, graph_offsets, k, mode, b.out, b.topk_idx, b.topk_score, b.workspace,
+                                    stream, fp32_path=fp32_path)
+    else:
+        rc = kmip_attn_forward(Q, K, V, graph_offsets, k, mode, b.out, b.topk_idx, b.topk_score, b.workspace, stream)
     if rc != KMIP_OK:
         raise KmipError(rc, "kmip_attn_forward")
     if check:

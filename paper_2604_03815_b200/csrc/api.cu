@@ -1,6 +1,7 @@
 // C ABI of the k-MIP attention library: argument validation and kernel sequencing.
 // Nothing here allocates device memory or synchronises the stream (kmip_last_status excepted).
 #include "common.cuh"
+#include "kmip_test.h"
 
 using namespace kmip;
 
@@ -28,7 +29,11 @@ struct Profile {
     cudaEvent_t bwd[kProfMaxCalls][4];
 };
 Profile g_prof;
-int g_fp32_path = 0;  // test hook, see kmip_debug_fp32_path
+
+int forward_impl(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G, int64_t N,
+                 int32_t H, int32_t d, int32_t k, int mode, float drop_p, uint64_t seed, void* out,
+                 int32_t* topk_idx, float* topk_score, void* workspace, size_t workspace_bytes, void* stream,
+                 const kmip_test_options_t* opt);
 
 }  // namespace
 
@@ -74,6 +79,26 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
                               int64_t N, int32_t H, int32_t d, int32_t k, int mode, float drop_p, uint64_t seed,
                               void* out, int32_t* topk_idx, float* topk_score, void* workspace,
                               size_t workspace_bytes, void* stream) {
+    return forward_impl(Q, K, V, graph_offsets, G, N, H, d, k, mode, drop_p, seed, out, topk_idx, topk_score, workspace,
+                        workspace_bytes, stream, nullptr);
+}
+
+int kmip_test_attn_forward(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
+                           int64_t N, int32_t H, int32_t d, int32_t k, int mode, void* out, int32_t* topk_idx,
+                           float* topk_score, void* workspace, size_t workspace_bytes, void* stream,
+                           const kmip_test_options_t* options) {
+    return forward_impl(Q, K, V, graph_offsets, G, N, H, d, k, mode, 0.0f, 0ull, out, topk_idx, topk_score, workspace,
+                        workspace_bytes, stream, options);
+}
+
+}  // extern "C"
+
+namespace {
+
+int forward_impl(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G, int64_t N,
+                 int32_t H, int32_t d, int32_t k, int mode, float drop_p, uint64_t seed, void* out,
+                 int32_t* topk_idx, float* topk_score, void* workspace, size_t workspace_bytes, void* stream,
+                 const kmip_test_options_t* opt) {
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
     if (!(drop_p >= 0.0f && drop_p < 1.0f)) return KMIP_ERR_INVALID_ARG;
@@ -91,6 +116,11 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
     a.drop_p = drop_p;
     a.seed = seed;
+    if (opt) {
+        a.wait_limit_cycles = opt->wait_limit_cycles;
+        a.drop_first_tile = opt->drop_first_tile;
+        a.fp32_path = opt->fp32_path;
+    }
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
@@ -98,7 +128,7 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
     // the tiled fp32 sweep runs one block per 128 query rows and head: worth it once that fills the GPU
     // about twice, below that the one-warp-per-row kernel has more parallelism
     const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k) &&
-                         (g_fp32_path == 0 ? (N / 128) * H >= 296 : g_fp32_path == 2);
+                         (a.fp32_path == 0 ? (N / 128) * H >= 2 * sm_count() : a.fp32_path == 2);
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.reorder && launch_reorder_queries(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.prune && (launch_reorder_keys(a, w) != cudaSuccess || launch_prune_stats(a, w) != cudaSuccess)) return KMIP_ERR_CUDA;
@@ -114,6 +144,10 @@ int kmip_attn_forward_dropout(const void* Q, const void* K, const void* V, const
     if (ev) cudaEventRecord(ev[4], a.stream);
     return KMIP_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 int kmip_attn_backward(const void* Q, const void* K, const void* V, const int32_t* graph_offsets, int32_t G,
                        int64_t N, int32_t H, int32_t d, int32_t k, int mode, const void* out, const void* d_out,
@@ -181,6 +215,15 @@ int kmip_last_status(const void* workspace, void* stream, int* device_status) {
     return KMIP_OK;
 }
 
+int kmip_attn_sweep_counters(const void* workspace, void* stream, int64_t* counters) {
+    if (!workspace || !counters) return KMIP_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;
+    StatusBlock sb;
+    if (cudaMemcpy(&sb, workspace, sizeof(sb), cudaMemcpyDeviceToHost) != cudaSuccess) return KMIP_ERR_CUDA;
+    for (int i = 0; i < 4; ++i) counters[i] = (int64_t)sb.counters[i];
+    return KMIP_OK;
+}
+
 int kmip_profile_enable(int max_calls) {
     if (g_prof.on) {
         for (int i = 0; i < g_prof.max_calls; ++i) {
@@ -227,26 +270,27 @@ int kmip_profile_read(double* stage_ms, int* calls) {
     return KMIP_OK;
 }
 
-// ---- test hook (not part of kmip.h): which fp32-mode sweep runs; 0 = by problem size, 1 = always one
-// warp per row, 2 = the tiled sweep whenever it supports (d, k), so that tests can put both on the same inputs
-void kmip_debug_fp32_path(int which) { g_fp32_path = which; }
-
-// ---- timing experiments (not part of kmip.h): see set_score_select_debug_flags
-void kmip_debug_set_flags(int flags) { set_score_select_debug_flags(flags); }
-// buf: device array of 8 * (number of SMs) int64, or NULL to switch off.  The pruned sweep writes, per CTA,
-// {key tiles of its work items, tiles it loaded (end-of-item markers included), (key tile, query tile)
-// pairs, pairs it scored}; debug builds of the full sweep write cycle counters there.
-void kmip_debug_set_timing(void* buf) { set_score_select_debug_timing(static_cast<long long*>(buf)); }
-
-// ---- test hook (not part of kmip.h): makes one bounded device-side wait run out, see score_select_tc.cu
-void kmip_debug_fault_test(int drop_first_tile, long long wait_limit_cycles) {
-    set_score_select_fault_test(drop_first_tile, wait_limit_cycles);
+int kmip_test_sweep_order(const void* workspace, int64_t N, int32_t G, int32_t H, int32_t d, int32_t k, int mode,
+                          int32_t* order, int32_t* rows_per_item, void* stream) {
+    const int rc = check_shape(N, H, d, k, mode);
+    if (rc != KMIP_OK) return rc;
+    if (!workspace || !order || !rows_per_item || G < 0) return KMIP_ERR_INVALID_ARG;
+    const bool tc = mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k);
+    const FwdWorkspace w = plan_fwd_workspace(N, G > 0 ? G : 1, H, d, tc, mode == KMIP_BF16_TC_PRUNED);
+    *rows_per_item = tc ? score_select_tc_rows_per_item(d, k) : 128;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (w.reorder) {
+        if (cudaMemcpy(order, static_cast<const unsigned char*>(workspace) + w.perm_off, (size_t)N * 4,
+                       cudaMemcpyDeviceToHost) != cudaSuccess)
+            return KMIP_ERR_CUDA;
+    } else {
+        for (int64_t i = 0; i < N; ++i) order[i] = (int32_t)i;
+    }
+    return KMIP_OK;
 }
 
-// ---- test hook (not part of kmip.h): dense scores of the tensor-core pipeline -----------------
-// Writes S[h][i][j] = q_i^h . k_j^h (fp32, [H, N, N]) for ONE graph of N <= 8192 nodes through the
-// same TMA / tcgen05 path as the forward pass, so tests can check the contraction element-wise.
-int kmip_debug_tc_scores(const void* Q, const void* K, int64_t N, int32_t H, int32_t d, float* scores,
+// Declared in kmip_test.h: dense scores of the tensor-core pipeline, for element-wise checks of the contraction.
+int kmip_test_tc_scores(const void* Q, const void* K, int64_t N, int32_t H, int32_t d, float* scores,
                          void* workspace, size_t workspace_bytes, void* stream) {
     const int rc = check_shape(N, H, d, 1, KMIP_BF16_TC);
     if (rc != KMIP_OK) return rc;

@@ -385,7 +385,7 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
 
     if ((err = cudaMemsetAsync(cursor, 0, sizeof(int) * (size_t)(n_rows + 1), a.stream)) != cudaSuccess) return err;
 
-    const int row_blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
+    const int row_blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 32);
     bwd_rows_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         K, V, dOut, a.topk_idx, a.topk_score, (int)a.N, a.H, a.k, scale, a.drop_p, a.seed, ws_p, ws_ds,
         static_cast<T*>(a.dQ));
@@ -402,7 +402,7 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
 
     bwd_segments_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         Q, dOut, seg_off, hits, n_rows, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
-    bwd_long_segments_kernel<T, D><<<148 * 8, kWarpsPerBlock * 32, 0, a.stream>>>(
+    bwd_long_segments_kernel<T, D><<<sm_count() * 8, kWarpsPerBlock * 32, 0, a.stream>>>(
         Q, dOut, seg_off, hits, long_list, sb, a.H, a.k, static_cast<T*>(a.dK), static_cast<T*>(a.dV));
     if (ev) cudaEventRecord(ev[2], a.stream);
     return cudaGetLastError();

@@ -21,7 +21,10 @@ struct StatusBlock {
     int detail;      // where it happened (kernel-specific code)
     int n_items;     // forward: number of work items the plan kernel produced
     int n_long;      // backward: number of long key segments
-    int reserved[60];
+    // pruned sweep: key tiles of all work items, tiles loaded (end-of-item markers included),
+    // (key tile, query tile) pairs, pairs scored - summed over the CTAs (kmip_attn_sweep_counters)
+    unsigned long long counters[4];
+    int reserved[52];
 };
 static_assert(sizeof(StatusBlock) == kStatusBytes, "status block size");
 
@@ -180,7 +183,13 @@ struct FwdArgs {
     cudaStream_t stream;
     float drop_p = 0.0f;             // attention dropout on the k weights (0 = none)
     unsigned long long seed = 0ull;  // of its counter-based draws
+    // per-call test options (kmip_test.h); the public entry points leave the defaults
+    long long wait_limit_cycles = 0;  // bound of every device-side wait in SM clocks; <= 0: kDefaultWaitLimitCycles
+    int drop_first_tile = 0;          // leave one key tile of CTA 0 unloaded, so that the waits on it run out
+    int fp32_path = 0;                // fp32 mode: 0 = sweep chosen by problem size, 1 = one warp per row, 2 = tiled
 };
+
+constexpr long long kDefaultWaitLimitCycles = 8000000000ll;  // about 4 s of SM clocks
 
 struct BwdArgs {
     const void *Q, *K, *V, *d_out;
@@ -210,13 +219,11 @@ cudaError_t launch_prune_stats(const FwdArgs& a, const FwdWorkspace& w);
 constexpr int kMinRowsToSort = 8192;  // smaller graphs keep their row and key order
 // score_select_exact.cu: CUDA-core scores + running top-k, any supported (d, k), fp32 or bf16 storage
 cudaError_t launch_score_select_exact(const FwdArgs& a);
+int sm_count();  // multiprocessors of the current device (cached per device)
 // score_select_tc.cu: tcgen05 scores + running top-k (bf16 storage); returns cudaErrorNotSupported
 // when (d, k) is outside what the tensor-core kernel covers
 bool score_select_tc_supported(int32_t d, int32_t k);
 int score_select_tc_rows_per_item(int32_t d, int32_t k);
-void set_score_select_debug_flags(int flags);
-void set_score_select_debug_timing(long long* buf);
-void set_score_select_fault_test(int drop_first_tile, long long wait_limit_cycles);
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump);
 // refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k

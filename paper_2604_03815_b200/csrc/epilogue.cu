@@ -43,7 +43,7 @@ softmax_gather_kernel(const T* __restrict__ V, const int32_t* __restrict__ topk_
 template <typename T, int D>
 cudaError_t launch_d(const FwdArgs& a) {
     const long long n_rows = (long long)a.N * a.H;
-    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
+    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 32);
     softmax_gather_kernel<T, D><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
         static_cast<const T*>(a.V), a.topk_idx, a.topk_score, (int)a.N, a.H, a.k,
         1.0f / sqrtf((float)a.d), a.drop_p, a.seed, static_cast<T*>(a.out), reinterpret_cast<const StatusBlock*>(a.ws));

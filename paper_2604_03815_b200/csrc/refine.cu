@@ -142,7 +142,7 @@ template <typename T, int D>
 cudaError_t launch_d(const FwdArgs& a, const T* keys, const int* kperm = nullptr) {
     constexpr bool REGROUPED = sizeof(T) == 2;
     const long long n_rows = (long long)a.N * a.H;
-    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 32);
+    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 32);
 #define KMIP_LAUNCH_REFINE(E_) \
     refine_topk_kernel<T, D, E_, REGROUPED><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
         static_cast<const T*>(a.Q), keys, a.graph_offsets, a.G, (int)a.N, a.H, a.k, \

@@ -377,12 +377,12 @@ cudaError_t launch_reorder_queries(const FwdArgs& a, const FwdWorkspace& w) {
         kern<<<w.max_items, kAssignThreads, smem, a.stream>>>(
             static_cast<const __nv_bfloat16*>(a.Q), static_cast<const __nv_bfloat16*>(a.K), HD,
             reinterpret_cast<const WorkItem*>(a.ws + w.items_off), sb, a.graph_offsets, a.G, nullptr, nullptr, code);
-        graph_sort_stable_kernel<kPivotBits><<<std::min(n_graphs, 148 * 2), kSortThreads, (32 << kPivotBits) * 4, a.stream>>>(
+        graph_sort_stable_kernel<kPivotBits><<<std::min(n_graphs, sm_count() * 2), kSortThreads, (32 << kPivotBits) * 4, a.stream>>>(
             a.graph_offsets, a.G, (int)a.N, code, perm, sb);
     } else {
         query_code_kernel<<<(unsigned)((a.N * 32 + 255) / 256), 256, 0, a.stream>>>(
             static_cast<const __nv_bfloat16*>(a.Q), (int)a.N, HD, code, sb);
-        graph_sort_kernel<kCodeBits><<<std::min(n_graphs, 148 * 2), kSortThreads, (1 << kCodeBits) * 4, a.stream>>>(
+        graph_sort_kernel<kCodeBits><<<std::min(n_graphs, sm_count() * 2), kSortThreads, (1 << kCodeBits) * 4, a.stream>>>(
             a.graph_offsets, a.G, (int)a.N, code, perm, sb);
     }
     const int vec_per_row = HD * 2 / 16;
@@ -421,7 +421,7 @@ cudaError_t launch_reorder_keys(const FwdArgs& a, const FwdWorkspace& w) {
     constexpr int sort_smem = (32 << kKeyCodeBits2) * 4;
     err = cudaFuncSetAttribute(sort, cudaFuncAttributeMaxDynamicSharedMemorySize, sort_smem);
     if (err != cudaSuccess) return err;
-    sort<<<std::min(n_graphs, 148 * 2), kSortThreads, sort_smem, a.stream>>>(a.graph_offsets, a.G, (int)a.N, code, kperm, sb);
+    sort<<<std::min(n_graphs, sm_count() * 2), kSortThreads, sort_smem, a.stream>>>(a.graph_offsets, a.G, (int)a.N, code, kperm, sb);
     const int vec_per_row = a.d * 2 / 16;
     const long long n_vec = (long long)a.N * a.H * vec_per_row;
     pack_keys_perm_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, a.stream>>>(

@@ -91,7 +91,7 @@ score_select_exact_kernel(const T* __restrict__ Q, const T* __restrict__ K,
 template <typename T, int D>
 cudaError_t launch_d(const FwdArgs& a) {
     const long long n_rows = (long long)a.N * a.H;
-    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 148LL * 64);
+    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 64);
     const T* Q = static_cast<const T*>(a.Q);
     const T* K = static_cast<const T*>(a.K);
     const dim3 grid(blocks), block(kWarpsPerBlock * 32);

@@ -184,7 +184,7 @@ cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w) {
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     const long long total = (long long)w.max_items * a.H;
-    const int grid = (int)std::min<long long>(total, 148LL * 16);
+    const int grid = (int)std::min<long long>(total, (long long)sm_count() * 16);
     kern<<<grid, ROWS, smem, a.stream>>>(static_cast<const float*>(a.Q), static_cast<const float*>(a.K),
                                          reinterpret_cast<const WorkItem*>(a.ws + w.items_off),
                                          reinterpret_cast<const StatusBlock*>(a.ws), a.H, a.k, a.topk_idx, a.topk_score);

@@ -43,13 +43,6 @@ namespace kmip {
 
 namespace {
 
-#ifndef KMIP_SWEEP_DEBUG
-#define KMIP_SWEEP_DEBUG 0
-#endif
-// Timing experiments (skip parts of the selection, per-role cycle counters) exist only in debug
-// builds; in the normal build `dbg` folds to 0 and none of the checks below reach the hot loop.
-constexpr bool kSweepDebug = KMIP_SWEEP_DEBUG != 0;
-
 constexpr int BM = 128;  // query rows per tile = TMEM lanes
 constexpr int BN = 128;  // keys per tile = accumulator columns
 constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -283,10 +276,9 @@ __global__ void __launch_bounds__(NQT * 128 + 96, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
-                       float* __restrict__ dump, int dump_ld /* = N */, int dbg_arg, long long* __restrict__ timing,
-                       long long wait_limit, int drop_first_tile, const int* __restrict__ perm, const PruneArgs pr) {
+                       float* __restrict__ dump, int dump_ld /* = N */, long long wait_limit, int drop_first_tile,
+                       const int* __restrict__ perm, const PruneArgs pr) {
     static_assert(!(DUMP && PRUNE), "the score dump sweeps every tile");
-    const int dbg = kSweepDebug ? dbg_arg : 0;
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
     constexpr int NEPI = 4 * NQT;
@@ -502,11 +494,11 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             kt = __shfl_sync(FULL, kt, 0);
             ++ic;
         }
-        if (timing && lane == 0) {  // per CTA: key tiles of its items, tiles loaded (with the end markers), pairs, pairs scored
-            timing[blockIdx.x * 8 + 0] = n_all;
-            timing[blockIdx.x * 8 + 1] = kt;
-            timing[blockIdx.x * 8 + 2] = n_pairs_all;
-            timing[blockIdx.x * 8 + 3] = n_pairs_live;
+        if (lane == 0) {  // key tiles of the CTA's items, tiles loaded (with the end markers), pairs, pairs scored
+            atomicAdd(&sb->counters[0], (unsigned long long)n_all);
+            atomicAdd(&sb->counters[1], (unsigned long long)kt);
+            atomicAdd(&sb->counters[2], (unsigned long long)n_pairs_all);
+            atomicAdd(&sb->counters[3], (unsigned long long)n_pairs_live);
         }
         if (!ok && lane == 0) {
             // give copies that are still in flight a bounded time to land before the CTA exits; a stage
@@ -580,7 +572,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
             int kt = 0, ic = 0;
             bool ok = true;
-            long long w_kfull = 0, w_tempty = 0, t_begin = clock64();
             for (long long w = blockIdx.x; ok && w < n_units; w += gridDim.x) {
                 int h_unused;
                 WorkItem it;
@@ -596,9 +587,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     // issuer (one query tile per CTA): a parity wait is sound only on a barrier whose
                     // every phase the waiter observes, and with an odd number of stages an issuer that
                     // skipped its partner's tiles would meet a stage only every second time it is filled.
-                    long long c0 = (dbg & 8) ? clock64() : 0;
                     if (!(ok = wait_or_abort<0>(bars.k_full(s), (kt / S) & 1, sAbort, sb, 4, wait_limit))) break;
-                    if (dbg & 8) w_kfull += clock64() - c0;
                     int tile_key = 0, tile_dead = 0;
                     if constexpr (PRUNE) {
                         tile_key = sStageKey[s];
@@ -610,9 +599,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         const int seq = kt * NQT + qt;
                         if ((seq & 1) != mine) continue;
                         const int b = seq & (NBUF - 1);
-                        long long c1 = (dbg & 8) ? clock64() : 0;
                         if (!(ok = wait_or_abort<0>(bars.t_empty(b), ((seq >> 2) & 1) ^ 1, sAbort, sb, 5, wait_limit))) break;
-                        if (dbg & 8) w_tempty += clock64() - c1;
                         ptx::tc_fence_after();
                         if constexpr (PRUNE) {
                             // a pair without scores (end of item, or ruled out for this query tile) still takes
@@ -642,12 +629,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 ptx::mma_commit(bars.q_empty());
                 ++ic;
             }
-            if ((dbg & 8) && timing && mine == 0) {
-                timing[blockIdx.x * 8 + 0] = clock64() - t_begin;
-                timing[blockIdx.x * 8 + 1] = w_kfull;
-                timing[blockIdx.x * 8 + 2] = w_tempty;
-                timing[blockIdx.x * 8 + 3] = kt;
-            }
             // all issued MMAs must have retired before tensor memory is released
             ptx::mma_commit(bars.done());
             const long long t0 = clock64();
@@ -668,8 +649,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         int flush_seen = 0;
         int tcnt = 0, ic = 0;
         bool ok = true;
-        long long w_tfull = 0, t_work = 0, t_begin = clock64();
-        long long prof[4] = {0, 0, 0, 0};
         for (long long w = blockIdx.x; ok && w < n_units; w += gridDim.x) {
             int h;
             WorkItem it;
@@ -733,12 +712,11 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     const int b = (tcnt * NQT + qt) & (NBUF - 1);
                     const uint32_t full_bar = full_bar0 + (uint32_t)b * (8u * NQT);
                     const uint32_t full_par = (uint32_t)(tcnt >> kUseShift) & 1u;
-                    const long long c0 = (dbg & 8) ? clock64() : 0;
                     if (!__all_sync(FULL, ptx::mbar_try_wait(full_bar, full_par))) {
                         // The scores are still not there after the try's own (hardware-bounded) wait:
                         // merge pending candidates into the lists meanwhile (always allowed, and it
                         // raises the thresholds early), then block.
-                        if (!(dbg & 3) && __any_sync(FULL, rs.cnt > 0)) {
+                        if (__any_sync(FULL, rs.cnt > 0)) {
                             flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
                             if constexpr (PRUNE) publish_thresholds(rs.tau, inv_qn, ic, warp_stat_s + 16u * warp, lane);
                         }
@@ -746,7 +724,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         ok = __all_sync(FULL, ok);
                         if (!ok) break;
                     }
-                    const long long c1 = (dbg & 8) ? clock64() : 0;
                     if constexpr (PRUNE) key0 = sBufKey[b];  // the tiles that arrive are not consecutive
                     // this query tile's MMAs on the key tile have retired; once that holds for every query
                     // tile the key stage can be refilled
@@ -767,49 +744,34 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                     float sub[16], quad[4];
                     uint32_t v[64];
                     ptx::tmem_ld_32x64_sync(taddr, v);
-                    if (!(dbg & 2)) {
-                        if (ragged) half_maxima<true>(v, ncol, sub, quad);
-                        else half_maxima<false>(v, BN, sub, quad);
-                    }
+                    if (ragged) half_maxima<true>(v, ncol, sub, quad);
+                    else half_maxima<false>(v, BN, sub, quad);
                     ptx::tmem_ld_32x64_sync(taddr + 64, v);
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
-                    if (!(dbg & 2)) {
-                        if (ragged) half_maxima<true>(v, ncol - 64, sub + 8, quad + 2);
-                        else half_maxima<false>(v, BN, sub + 8, quad + 2);
-                        const float gm = fmaxf(fmaxf(quad[0], quad[1]), fmaxf(quad[2], quad[3]));
-                        if (!(dbg & 1)) {
-                            const long long p0 = (dbg & 8) ? clock64() : 0;
-                            // A flush by one warp stalls the others within a few tiles (the accumulator ring
-                            // is only four deep), so the warps flush together: whoever must flush bumps a
-                            // CTA-wide counter and every warp that sees it move flushes at its next tile.
-                            const int req = (int)ptx::lds_u32(flush_req_s);
-                            bool do_flush = req != flush_seen;
-                            if (__any_sync(FULL, gm > rs.tau)) {  // some lane of the warp has a hit in this tile
-                                uint32_t pend = wp_addr + (uint32_t)rs.cnt * 256u;
-                                append_groups(sub, quad, rs.tau, key0, pend);
-                                rs.cnt = (int)((pend - wp_addr) >> 8);
-                                if (dbg & 8) { prof[0] += clock64() - p0; ++prof[1]; }
-                                if (__any_sync(FULL, rs.cnt > ROOM - 16)) {  // a tile adds at most 16 groups per row
-                                    do_flush = true;
-                                    if (lane == 0 && req == flush_seen) atomicAdd(const_cast<int*>(sFlushReq), 1);
-                                }
-                            }
-                            if (do_flush) {
-                                const long long p1 = (dbg & 8) ? clock64() : 0;
-                                flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
-                                if constexpr (PRUNE) publish_thresholds(rs.tau, inv_qn, ic, warp_stat_s + 16u * warp, lane);
-                                flush_seen = req + ((req == flush_seen) ? 1 : 0);
-                                if (dbg & 8) { prof[2] += clock64() - p1; ++prof[3]; }
-                            }
-                        } else if (gm == 123.456f) {
-                            rs.tau = 0.0f;  // timing experiment: keep the maxima alive
+                    if (ragged) half_maxima<true>(v, ncol - 64, sub + 8, quad + 2);
+                    else half_maxima<false>(v, BN, sub + 8, quad + 2);
+                    const float gm = fmaxf(fmaxf(quad[0], quad[1]), fmaxf(quad[2], quad[3]));
+                    // A flush by one warp stalls the others within a few tiles (the accumulator ring
+                    // is only four deep), so the warps flush together: whoever must flush bumps a
+                    // CTA-wide counter and every warp that sees it move flushes at its next tile.
+                    const int req = (int)ptx::lds_u32(flush_req_s);
+                    bool do_flush = req != flush_seen;
+                    if (__any_sync(FULL, gm > rs.tau)) {  // some lane of the warp has a hit in this tile
+                        uint32_t pend = wp_addr + (uint32_t)rs.cnt * 256u;
+                        append_groups(sub, quad, rs.tau, key0, pend);
+                        rs.cnt = (int)((pend - wp_addr) >> 8);
+                        if (__any_sync(FULL, rs.cnt > ROOM - 16)) {  // a tile adds at most 16 groups per row
+                            do_flush = true;
+                            if (lane == 0 && req == flush_seen) atomicAdd(const_cast<int*>(sFlushReq), 1);
                         }
-                    } else if (v[0] == 0x12345678u && v[63] == 1u) {
-                        rs.tau = 0.0f;  // timing experiment: keep the loads alive
                     }
-                    if (dbg & 8) { w_tfull += c1 - c0; t_work += clock64() - c1; }
+                    if (do_flush) {
+                        flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
+                        if constexpr (PRUNE) publish_thresholds(rs.tau, inv_qn, ic, warp_stat_s + 16u * warp, lane);
+                        flush_seen = req + ((req == flush_seen) ? 1 : 0);
+                    }
                 }
             }
             if (!ok) break;
@@ -832,13 +794,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
             ++ic;
         }
-        if ((dbg & 8) && timing && threadIdx.x == 0) {
-            timing[blockIdx.x * 8 + 4] = clock64() - t_begin;
-            timing[blockIdx.x * 8 + 5] = w_tfull;
-            timing[blockIdx.x * 8 + 6] = t_work;
-            timing[blockIdx.x * 8 + 7] = tcnt;
-            for (int i = 0; i < 4; ++i) timing[148 * 8 + blockIdx.x * 8 + i] = prof[i];
-        }
     }
 
     ptx::tc_fence_before();
@@ -850,11 +805,6 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 }
 
 // ------------------------------------------------------------------------------------------- host
-int g_debug_flags = 0;  // timing experiments only (see set_score_select_debug_flags)
-long long* g_debug_timing = nullptr;
-long long g_wait_limit_cycles = 8000000000ll;  // bound of every device-side wait, in SM clocks (about 4 s)
-int g_drop_first_tile = 0;                     // failure-detection test hook, see set_score_select_fault_test  // device buffer [grid][8] of cycle counters when flag bit 3 is set
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -890,18 +840,6 @@ bool make_tensor_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t ro
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-    static int sms[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (sms[dev] == 0) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
-        sms[dev] = v;
-    }
-    return sms[dev];
-}
-
 template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE>
 cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     using Sh = TcShape<D>;
@@ -924,8 +862,8 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     const int grid = (int)std::min<long long>(sm_count(), max_total);
     kern<<<grid, NQT * 128 + 96, smem_bytes, a.stream>>>(
         tmQ, tmK, reinterpret_cast<const WorkItem*>(a.ws + w.items_off), reinterpret_cast<StatusBlock*>(a.ws),
-        a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, g_debug_flags, g_debug_timing, g_wait_limit_cycles,
-        g_drop_first_tile, (w.reorder && !DUMP) ? reinterpret_cast<const int*>(a.ws + w.perm_off) : nullptr, pr);
+        a.H, a.k, a.topk_idx, a.topk_score, dump, (int)a.N, a.wait_limit_cycles > 0 ? a.wait_limit_cycles : kDefaultWaitLimitCycles,
+        a.drop_first_tile, (w.reorder && !DUMP) ? reinterpret_cast<const int*>(a.ws + w.perm_off) : nullptr, pr);
     return cudaGetLastError();
 }
 
@@ -959,16 +897,16 @@ cudaError_t launch_any(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
 
 }  // namespace
 
-// bit 0: skip the candidate path, bit 1: skip the whole filter.  Results are then meaningless;
-// used only to time the tensor pipeline and the tensor-memory loads in isolation.
-void set_score_select_debug_flags(int flags) { g_debug_flags = flags; }
-void set_score_select_debug_timing(long long* buf) { g_debug_timing = buf; }
-
-// Test hook for the bounded waits: with drop_first_tile != 0 the next launches leave one key tile of
-// CTA 0 unloaded (a wait that nothing will ever satisfy); wait_limit_cycles <= 0 restores the default.
-void set_score_select_fault_test(int drop_first_tile, long long wait_limit_cycles) {
-    g_drop_first_tile = drop_first_tile;
-    g_wait_limit_cycles = wait_limit_cycles > 0 ? wait_limit_cycles : 8000000000ll;
+int sm_count() {
+    static int sms[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (sms[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        sms[dev] = v;
+    }
+    return sms[dev];
 }
 
 bool score_select_tc_supported(int32_t d, int32_t k) {

@@ -44,7 +44,13 @@ extern "C" int kmip_attn_forward_static_scratch(const void* Q, const void* K, co
     const int rc = kmip_attn_workspace_bytes(N, graph_offsets ? G : 1, H, d, k, mode, KMIP_PASS_FORWARD, &need);
     if (rc != KMIP_OK) return rc;
     if (need > kStaticScratchBytes) return KMIP_ERR_TOO_LARGE;
-    if (N == 0) return KMIP_OK;
+    if (N == 0) {
+        // nothing to enqueue, but a caller that polls device_status must not read the previous call's word
+        if (device_status != nullptr &&
+            cudaMemsetAsync(device_status, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return KMIP_ERR_CUDA;
+        return KMIP_OK;
+    }
     void* scratch = scratch_address_for_current_device();
     if (scratch == nullptr) return KMIP_ERR_CUDA;
     // The regular entry point clears the status block and rewrites the work items and the regrouped

@@ -1,4 +1,4 @@
-// Diagnostic of the paper's App. H ("cumulative attention weight"): the share of the FULL softmax
+// Diagnostic of the paper's App. I ("cumulative attention weight"): the share of the FULL softmax
 // over all keys of the query's graph that falls on the k keys the forward pass kept,
 //   mass[i,h] = sum_t exp(s_t / sqrt(d)) / sum_j exp(q_i . k_j / sqrt(d)),   s = topk_score[i,h,:].
 // The denominator needs every score of the row again; they are computed on CUDA cores in fp32
@@ -101,7 +101,7 @@ topk_mass_kernel(const T* __restrict__ Q, const T* __restrict__ K, const WorkIte
 template <typename T, int D>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* mass) {
     const long long total = (long long)w.max_items * a.H;
-    const int grid = (int)std::min<long long>(total, 148LL * 16);
+    const int grid = (int)std::min<long long>(total, (long long)sm_count() * 16);
     topk_mass_kernel<T, D><<<grid, ROWS, 0, a.stream>>>(
         static_cast<const T*>(a.Q), static_cast<const T*>(a.K), reinterpret_cast<const WorkItem*>(a.ws + w.items_off),
         reinterpret_cast<const StatusBlock*>(a.ws), a.H, a.k, a.topk_score, mass);

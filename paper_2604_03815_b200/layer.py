@@ -28,6 +28,12 @@ class KMIPAttentionFunction(torch.autograd.Function):
                                           fb.topk_score, fb.workspace)
         if rc != kb.KMIP_OK:
             raise kb.KmipError(rc, "kmip_attn_forward_dropout")
+        if not any(ctx.needs_input_grad[:3]):
+            # no backward call will follow (eval, no_grad), so a device-side problem (malformed offsets, an
+            # expired bounded wait) has to surface here: the kernels after it leave `out` unwritten
+            st = kb.kmip_last_status(fb.workspace)
+            if st != kb.KMIP_OK:
+                raise kb.KmipError(st, "kmip_attn_forward (device)")
         ctx.save_for_backward(Q, K, V, fb.out, fb.topk_idx, fb.topk_score)
         ctx.graph_offsets, ctx.k, ctx.mode, ctx.fwd_workspace = graph_offsets, k, mode, fb.workspace
         ctx.drop_p, ctx.seed = drop_p, seed

@@ -1,4 +1,4 @@
-"""The paper's controlled size sweep (Sec. 5 "Objective 1", App. G.2 and the tables of App. H.1 / I)
+"""The paper's controlled size sweep (Sec. 5 "Objective 1", App. H.2 and the tables of App. J.1 / K)
 on this library: one (N x d_K) Q/K/V triple with d_K = 10 and k = 10, normal inputs, time of an
 inference pass (forward) and of a training pass (forward + backward) and peak device memory, for
 N = 10^(i/2).  The library stores head widths 16/32/64/128, so d_K = 10 is zero-padded to 16.
@@ -6,7 +6,7 @@ N = 10^(i/2).  The library stores head widths 16/32/64/128, so d_K = 10 is zero-
     python -m paper_2604_03815_b200.paper_sweep [--min-exp 8] [--max-exp 13] [--mode bf16|fp32] [--reps 3]
 
 Prints one JSON line per size and a markdown table at the end.  The paper's own figures (A100-40GB,
-fp32 on CUDA cores, Tables of App. H.1 / I) are printed beside ours as context: another GPU,
+fp32 on CUDA cores, Tables of App. J.1 / K) are printed beside ours as context: another GPU,
 another precision, not a target.
 """
 import argparse
@@ -17,7 +17,7 @@ import numpy as np
 from . import binding as kb
 from . import workloads as wl
 
-# N -> (inference seconds, training seconds) reported by the paper for k-MIP attention (App. H.1, App. I)
+# N -> (inference seconds, training seconds) reported by the paper for k-MIP attention (App. J.1, App. K)
 PAPER_SECONDS = {
     10 ** 4: (3.14e-3, None), 31623: (6.38e-3, 8.46e-3), 10 ** 5: (34.45e-3, 39.94e-3),
     316228: (0.231, 0.245), 10 ** 6: (2.146, 2.233), 3162278: (20.966, 21.232), 10 ** 7: (None, 208.338),

@@ -16,7 +16,7 @@ out, and returned as float32 (a bf16 value is exactly representable in float32),
 so the fp32 path, the bf16 path and the fp64 oracle all see the same real numbers.
 
 The five workloads mirror the shapes of the paper's experiments (Sec. 5,
-App. G: batched small graphs of a few hundred nodes, single city-scale graphs
+App. H: batched small graphs of a few hundred nodes, single city-scale graphs
 of 1e5..5e5 nodes, 4-8 heads, k between 5 and 45) with synthetic values.
 """
 from __future__ import annotations

@@ -29,6 +29,11 @@ def test_exports_every_declared_symbol(kb):
     L = kb.lib()
     for n in set(names):
         assert hasattr(L, n), f"{n} is declared in include/ but not exported"
+    # and the other direction: the library exports no kmip_* symbol that no header declares
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", kb.LIB_PATH], capture_output=True, text=True, check=True).stdout
+    exported = {ln.split()[-1] for ln in out.splitlines() if ln.split() and ln.split()[-1].startswith("kmip_")}
+    assert exported == set(names), f"undeclared exports: {sorted(exported - set(names))}"
 
 
 def test_version_and_status_strings(kb):

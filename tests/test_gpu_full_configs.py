@@ -1,7 +1,9 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration bench.py times.
-The oracle brute-forces a seeded, stratified sample of query rows against all keys of their
-graph (selection, scores, outputs); the backward oracle, which is linear in N, runs in full on
-the GPU's validated index set."""
+The oracle brute-forces a seeded, stratified sample of at least 4096 query rows against all keys of
+their graph (selection, scores, outputs) - stratified by the row's place in the sweep (work-item and
+query-tile borders in sweep order, whole work items of the schedule's split tail), by cluster and by
+hub / non-hub, see parity_util.stratified_rows; the backward oracle, which is linear in N, runs in
+full on the GPU's validated index set."""
 import numpy as np
 import pytest
 import torch
@@ -18,8 +20,10 @@ def _full(cfg, n_sample):
     w = wl.make_config(cfg)
     dev = pu.to_device(w)
     fb = pu.run_forward(w, dev)
-    rows = wl.sample_rows(w, n_sample)
+    rows, info = pu.stratified_rows(w, fb, n_sample)
+    assert len(rows) >= n_sample
     st = pu.check_forward(w, fb, rows)
+    st.update(info)
     # every row: structure checks that hold at any size
     idx = fb.topk_idx.cpu().numpy()
     offs = w.graph_offsets.astype(np.int64)
@@ -33,17 +37,18 @@ def _full(cfg, n_sample):
 
 
 def test_config3_100k_nodes():
-    st = _full(3, 384)
+    st = _full(3, 4096)
     assert st["identical_rows"] > 0.99
 
 
 def test_config4_500k_point_cloud():
-    st = _full(4, 256)
+    st = _full(4, 4096)
     assert st["identical_rows"] > 0.95
+    assert st["tail_items"] >= 4        # the sample holds whole work items of the schedule's split tail
 
 
 def test_config5_hub_batch():
-    st = _full(5, 256)
+    st = _full(5, 4096)
     assert st["identical_rows"] > 0.95
 
 

@@ -103,3 +103,23 @@ def test_layer_attention_dropout_only_in_training():
     xg = x.clone().requires_grad_(True)
     layer(xg).float().square().sum().backward()
     assert torch.isfinite(xg.grad.float()).all() and float(xg.grad.float().abs().max()) > 0
+
+
+def test_forward_only_use_surfaces_device_errors():
+    """Under torch.no_grad() no backward call follows, so malformed graph offsets (seen only by the
+    device) must raise from the forward call instead of handing back unwritten memory."""
+    from paper_2604_03815_b200 import binding as kb
+    from paper_2604_03815_b200.layer import KMIPSelfAttention
+
+    torch.manual_seed(7)
+    layer = KMIPSelfAttention(32, 2, 16, 4, dtype=torch.bfloat16)
+    x = torch.randn(600, 32, device="cuda").to(torch.bfloat16)
+    bad = torch.tensor([0, 400, 300, 600], dtype=torch.int32, device="cuda")
+    with torch.no_grad():
+        with pytest.raises(kb.KmipError) as e:
+            layer(x, bad)
+    assert e.value.status == kb.KMIP_ERR_BAD_OFFSETS
+    good = torch.tensor([0, 300, 600], dtype=torch.int32, device="cuda")
+    with torch.no_grad():
+        y = layer(x, good)          # the context is still usable
+    assert torch.isfinite(y.float()).all()

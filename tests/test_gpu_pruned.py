@@ -25,7 +25,8 @@ def _check(w, n_sample, backward=True):
     w = _pruned(w)
     dev = pu.to_device(w)
     fb = pu.run_forward(w, dev)
-    st = pu.check_forward(w, fb, wl.sample_rows(w, n_sample))
+    rows = pu.stratified_rows(w, fb, n_sample)[0] if n_sample >= 4096 else wl.sample_rows(w, n_sample)
+    st = pu.check_forward(w, fb, rows)
     idx = fb.topk_idx.cpu().numpy()
     sc = fb.topk_score.cpu().numpy()
     offs = w.graph_offsets.astype(np.int64)
@@ -91,12 +92,12 @@ def test_same_answer_as_the_full_sweep():
 
 
 def test_config4_500k_point_cloud_pruned():
-    st = _check(wl.make_config(4), 256)
+    st = _check(wl.make_config(4), 4096)
     assert st["identical_rows"] > 0.95
 
 
 def test_config5_hub_batch_pruned():
-    st = _check(wl.make_config(5), 256)
+    st = _check(wl.make_config(5), 4096)
     assert st["identical_rows"] > 0.95
 
 

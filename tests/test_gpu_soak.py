@@ -101,14 +101,10 @@ def test_random_small_shapes_against_the_oracle():
         mode = wl.MODE_BF16_TC if rng.random() < 0.7 else wl.MODE_FP32_EXACT
         path = int(rng.integers(0, 3)) if mode == wl.MODE_FP32_EXACT else 0
         w = wl.iid_workload("s", 700000 + case, sizes, H, d, k, mode, input_scale=float(rng.choice([0.2, 1.0])) / np.sqrt(d))
-        kb.lib().kmip_debug_fp32_path(path)
-        try:
-            dev = pu.to_device(w)
-            fb = pu.run_forward(w, dev)
-            pu.check_forward(w, fb)
-            pu.check_backward(w, fb, pu.run_backward(w, fb, dev))
-        finally:
-            kb.lib().kmip_debug_fp32_path(0)
+        dev = pu.to_device(w)
+        fb = pu.run_forward(w, dev, fp32_path=path)
+        pu.check_forward(w, fb)
+        pu.check_backward(w, fb, pu.run_backward(w, fb, dev))
 
 
 def _pruned_case(rng, case, seed):

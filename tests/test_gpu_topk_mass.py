@@ -1,4 +1,4 @@
-"""The cumulative-attention-weight diagnostic (App. H): the CUDA path against the oracle's plain
+"""The cumulative-attention-weight diagnostic (App. I): the CUDA path against the oracle's plain
 definition (all scores, full softmax, sum of the k largest probabilities)."""
 import numpy as np
 import pytest
