@@ -220,12 +220,15 @@ int kmip_attn_forward_static_scratch(const void *Q, const void *K, const void *V
 int kmip_last_status(const void *workspace, void *stream, int *device_status);
 
 /*
- * Work counters of the pruned sweep (KMIP_BF16_TC_PRUNED; the paper has no counterpart).  Synchronises
- * `stream`, then reads from the status block of `workspace` (the forward workspace of the last
- * call) counters[4] = {key tiles of all work items, key tiles loaded (one end marker per work item
- * included), (key tile, query tile) pairs, pairs scored}, summed over the sweep's CTAs.  All zero
- * after a call in another mode.  counters: HOST memory, four int64.  Returns KMIP_ERR_CUDA if the
- * synchronisation or the copy fails.
+ * Work counters of the last forward call on `workspace` (the paper has no counterpart).  Synchronises
+ * `stream`, then reads from the status block of `workspace` into counters[8] (HOST memory, int64):
+ *   [0..3]  KMIP_BF16_TC_PRUNED: key tiles of all work items, key tiles loaded (one end marker per work
+ *           item included), (key tile, query tile) pairs, pairs scored, summed over the sweep's CTAs;
+ *   [4]     KMIP_BF16_TC with d <= 32 and k <= 32: (query, head) pairs that the half-precision prefilter
+ *           could not decide and the exact kernel recomputed from all keys;
+ *   [5..7]  zero.
+ * Counters of a path that did not run are zero.  Returns KMIP_ERR_CUDA if the synchronisation or the
+ * copy fails.
  */
 int kmip_attn_sweep_counters(const void *workspace, void *stream, int64_t *counters);
 

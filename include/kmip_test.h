@@ -52,6 +52,19 @@ int kmip_test_tc_scores(const void *Q, const void *K, int64_t N, int32_t H, int3
                         float *scores, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The scores of the half-precision prefilter sweep (head widths 16 and 32): the tensor-core contraction of
+ * the scaled fp16 copies of Q and K with fp16 accumulators, T[h][i][j] ~ s_q[h] s_k[h] (q_i^h . k_j^h), written
+ * as fp32 [H, N, N] to `scores` for ONE graph of 1 <= N <= 8192 nodes.  `stats` (device, float [H, 4]) receives
+ * per head {largest squared query-row norm, largest squared key-row norm, largest squared norm of the first
+ * 16 elements of a key row, 0} as the conversion measured them; the scales s_q, s_k are the powers of two that
+ * put the largest norm into [32, 64).  Tests use it to check the error bound the rescoring kernel relies on.
+ * workspace: kmip_attn_workspace_bytes(N, 1, H, d, 1, KMIP_BF16_TC, KMIP_PASS_FORWARD) bytes.
+ * d > 32 is KMIP_ERR_UNSUPPORTED; other errors as for kmip_test_tc_scores.
+ */
+int kmip_test_f16_scores(const void *Q, const void *K, int64_t N, int32_t H, int32_t d,
+                         float *scores, float *stats, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Where the tensor-core sweep of the last kmip_attn_forward call on `workspace` put each query row,
  * so that tests can sample rows by their place in the sweep (work-item borders, the split tail of
  * the schedule) and not only by their row number.  Synchronises `stream`, then writes to HOST memory

@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
         # kmip_test.h
         L.kmip_test_tc_scores.restype = ctypes.c_int
         L.kmip_test_tc_scores.argtypes = [P, P, i64, i32, i32, P, P, sz, P]
+        L.kmip_test_f16_scores.restype = ctypes.c_int
+        L.kmip_test_f16_scores.argtypes = [P, P, i64, i32, i32, P, P, P, sz, P]
         L.kmip_test_sweep_order.restype = ctypes.c_int
         L.kmip_test_sweep_order.argtypes = [P, i64, i32, i32, i32, i32, ctypes.c_int, P, ctypes.POINTER(i32), P]
         L.kmip_test_attn_forward.restype = ctypes.c_int
@@ -220,6 +222,13 @@ def kmip_test_tc_scores(Q, K, scores, workspace, stream=None) -> int:
                                          workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
+def kmip_test_f16_scores(Q, K, scores, stats, workspace, stream=None) -> int:
+    """kmip_test.h: scaled fp16-accumulated scores [H, N, N] of one small graph and the per-head statistics [H, 4]."""
+    N, H, d = Q.shape
+    return int(lib().kmip_test_f16_scores(_ptr(Q), _ptr(K), N, H, d, _ptr(scores), _ptr(stats), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
 def kmip_test_attn_forward(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score, workspace, stream=None,
                            wait_limit_cycles=0, drop_first_tile=0, fp32_path=0) -> int:
     """kmip_test.h: the forward pass with per-call test options; returns the library's status code."""
@@ -246,9 +255,10 @@ def kmip_test_sweep_order(workspace, N, G, H, d, k, mode, stream=None):
 
 
 def kmip_attn_sweep_counters(workspace, stream=None):
-    """Work counters of the pruned sweep's last call on `workspace` (synchronises the stream):
-    (key tiles, key tiles loaded, (key tile, query tile) pairs, pairs scored)."""
-    c = (ctypes.c_int64 * 4)()
+    """Work counters of the last forward call on `workspace` (synchronises the stream): (key tiles, key tiles
+    loaded, (key tile, query tile) pairs, pairs scored) of the pruned sweep, then the rows the half-precision
+    prefilter handed to the exact kernel, then three zeros."""
+    c = (ctypes.c_int64 * 8)()
     rc = lib().kmip_attn_sweep_counters(_ptr(workspace), _stream(stream), c)
     if rc != KMIP_OK:
         raise KmipError(rc, "kmip_attn_sweep_counters")

@@ -61,8 +61,7 @@ int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
     if (pass == KMIP_PASS_FORWARD)
-        *bytes = plan_fwd_workspace(N, G, H, d, mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k),
-                                    mode == KMIP_BF16_TC_PRUNED).total;
+        *bytes = plan_fwd_workspace(N, G, H, d, k, mode).total;
     else if (pass == KMIP_PASS_BACKWARD) *bytes = plan_bwd_workspace(N, H, k).total;
     else return KMIP_ERR_INVALID_ARG;
     return KMIP_OK;
@@ -108,8 +107,8 @@ int forward_impl(const void* Q, const void* K, const void* V, const int32_t* gra
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || !aligned16(topk_idx) ||
         !aligned16(topk_score) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
         return KMIP_ERR_INVALID_ARG;
-    const bool tc = mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k);
-    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, tc, mode == KMIP_BF16_TC_PRUNED);
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, k, mode);
+    const bool tc = w.tc;
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
 
     FwdArgs a{Q, K, V, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, out, topk_idx, topk_score,
@@ -124,20 +123,23 @@ int forward_impl(const void* Q, const void* K, const void* V, const int32_t* gra
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
-    if (tc && !w.prune && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (tc && !w.prune && !w.f16 && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     // the tiled fp32 sweep runs one block per 128 query rows and head: worth it once that fills the GPU
     // about twice, below that the one-warp-per-row kernel has more parallelism
     const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k) &&
                          (a.fp32_path == 0 ? (N / 128) * H >= 2 * sm_count() : a.fp32_path == 2);
     if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.reorder && launch_reorder_queries(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (w.f16 && launch_f16_convert(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.prune && (launch_reorder_keys(a, w) != cudaSuccess || launch_prune_stats(a, w) != cudaSuccess)) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], a.stream);
-    const cudaError_t sweep = tc ? launch_score_select_tc(a, w)
+    const cudaError_t sweep = w.f16 ? launch_score_select_f16(a, w) : tc ? launch_score_select_tc(a, w)
                               : tiled32 ? launch_score_select_fp32_tiled(a, w) : launch_score_select_exact(a);
     if (sweep != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], a.stream);
-    if (tc && launch_refine_topk(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (w.f16 && (launch_refine_f16(a, w) != cudaSuccess || launch_score_select_exact_redo(a, w) != cudaSuccess))
+        return KMIP_ERR_CUDA;
+    if (tc && !w.f16 && launch_refine_topk(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (tiled32 && launch_refine_topk_fp32(a) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[3], a.stream);
     if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
@@ -196,7 +198,7 @@ int kmip_attn_topk_mass(const void* Q, const void* K, const int32_t* graph_offse
     if (!aligned16(Q) || !aligned16(K) || !aligned16(topk_score) || !aligned16(workspace) ||
         (reinterpret_cast<uintptr_t>(mass) & 3u) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
         return KMIP_ERR_INVALID_ARG;
-    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, false);
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, k, mode, kPlanNoTensorCore);
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
     FwdArgs a{Q, K, nullptr, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, nullptr, nullptr,
               const_cast<float*>(topk_score), static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
@@ -221,6 +223,8 @@ int kmip_attn_sweep_counters(const void* workspace, void* stream, int64_t* count
     StatusBlock sb;
     if (cudaMemcpy(&sb, workspace, sizeof(sb), cudaMemcpyDeviceToHost) != cudaSuccess) return KMIP_ERR_CUDA;
     for (int i = 0; i < 4; ++i) counters[i] = (int64_t)sb.counters[i];
+    counters[4] = sb.n_redo;
+    counters[5] = counters[6] = counters[7] = 0;
     return KMIP_OK;
 }
 
@@ -275,9 +279,8 @@ int kmip_test_sweep_order(const void* workspace, int64_t N, int32_t G, int32_t H
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
     if (!workspace || !order || !rows_per_item || G < 0) return KMIP_ERR_INVALID_ARG;
-    const bool tc = mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k);
-    const FwdWorkspace w = plan_fwd_workspace(N, G > 0 ? G : 1, H, d, tc, mode == KMIP_BF16_TC_PRUNED);
-    *rows_per_item = tc ? score_select_tc_rows_per_item(d, k) : 128;
+    const FwdWorkspace w = plan_fwd_workspace(N, G > 0 ? G : 1, H, d, k, mode);
+    *rows_per_item = w.tc ? score_select_tc_rows_per_item(d, k) : 128;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.reorder) {
         if (cudaMemcpy(order, static_cast<const unsigned char*>(workspace) + w.perm_off, (size_t)N * 4,
@@ -295,7 +298,7 @@ int kmip_test_tc_scores(const void* Q, const void* K, int64_t N, int32_t H, int3
     const int rc = check_shape(N, H, d, 1, KMIP_BF16_TC);
     if (rc != KMIP_OK) return rc;
     if (!Q || !K || !scores || !workspace || N < 1 || N > 8192) return KMIP_ERR_INVALID_ARG;
-    const FwdWorkspace w = plan_fwd_workspace(N, 1, H, d, true);
+    const FwdWorkspace w = plan_fwd_workspace(N, 1, H, d, 1, KMIP_BF16_TC, kPlanTcFp32Acc);
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
     FwdArgs a{Q, K, nullptr, nullptr, 1, N, H, d, 1, KMIP_BF16_TC, nullptr, nullptr, nullptr,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
@@ -303,6 +306,27 @@ int kmip_test_tc_scores(const void* Q, const void* K, int64_t N, int32_t H, int3
     if (launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_plan(a, w, score_select_tc_rows_per_item(d, 1)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_score_dump_tc(a, w, scores) != cudaSuccess) return KMIP_ERR_CUDA;
+    return KMIP_OK;
+}
+
+int kmip_test_f16_scores(const void* Q, const void* K, int64_t N, int32_t H, int32_t d, float* scores, float* scales,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_shape(N, H, d, 1, KMIP_BF16_TC);
+    if (rc != KMIP_OK) return rc;
+    if (d > 32) return KMIP_ERR_UNSUPPORTED;
+    if (!Q || !K || !scores || !scales || !workspace || N < 1 || N > 8192) return KMIP_ERR_INVALID_ARG;
+    const FwdWorkspace w = plan_fwd_workspace(N, 1, H, d, 1, KMIP_BF16_TC, kPlanTcFp16Acc);
+    if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
+    FwdArgs a{Q, K, nullptr, nullptr, 1, N, H, d, 1, KMIP_BF16_TC, nullptr, nullptr, nullptr,
+              static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
+    if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_plan(a, w, score_select_tc_rows_per_item(d, 1)) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_f16_convert(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_score_dump_f16(a, w, scores) != cudaSuccess) return KMIP_ERR_CUDA;
+    // per head: {q_n2max, k_n2max, k_first16_n2max, 0} as the conversion measured them
+    if (cudaMemcpyAsync(scales, a.ws + w.f16stat_off, sizeof(float) * 4 * (size_t)H, cudaMemcpyDeviceToDevice, a.stream) !=
+        cudaSuccess)
+        return KMIP_ERR_CUDA;
     return KMIP_OK;
 }
 

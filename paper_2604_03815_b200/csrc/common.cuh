@@ -24,7 +24,8 @@ struct StatusBlock {
     // pruned sweep: key tiles of all work items, tiles loaded (end-of-item markers included),
     // (key tile, query tile) pairs, pairs scored - summed over the CTAs (kmip_attn_sweep_counters)
     unsigned long long counters[4];
-    int reserved[52];
+    int n_redo;      // forward, fp16 prefilter: rows the rescoring kernel sent to the exact kernel
+    int reserved[51];
 };
 static_assert(sizeof(StatusBlock) == kStatusBytes, "status block size");
 
@@ -42,8 +43,10 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a = kAlign) { return
 
 struct FwdWorkspace {
     size_t items_off;  // WorkItem[max_items]
-    size_t kpack_off;  // bf16 [H, N, d]: K regrouped by head for the tensor-core sweep (0 bytes otherwise)
-    size_t qperm_off;  // bf16 [N, H, d]: Q in the sweep's row order (only when `reorder`)
+    size_t kpack_off;  // [H, N, d], 2 bytes per element: K regrouped by head for the tensor-core sweeps (bf16, or
+                       // scaled fp16 for the half-precision prefilter; 0 bytes without a tensor-core sweep)
+    size_t qperm_off;  // [N, H, d], 2 bytes per element: Q in the sweep's row order (bf16, only when `reorder`;
+                       // scaled fp16 whenever `f16`)
     size_t perm_off;   // int  [N]: original row of each sweep row
     size_t code_off;   // u16  [N]: locality codes of the query rows
     // pruned sweep only (all 0 bytes otherwise):
@@ -55,27 +58,47 @@ struct FwdWorkspace {
     size_t qnorm_off;   // float [N, H]: norm of each query row's head slice, in sweep order
     size_t qstat_off;   // float [max_items, 3, H, d+4]: centroid, radius, centroid norm of each item's 128-row query tiles
     size_t kstat_off;   // float [max_tiles, H, d+4]: centroid, radius, centroid norm, largest norm of each key tile
+    // half-precision prefilter only (all 0 bytes otherwise):
+    size_t f16stat_off;    // F16HeadStat [H]: per-head norm maxima
+    size_t cand_word_off;  // u32 [N, H, list]: the groups each row kept (first key of the 16-key window, bit 31 = odd keys)
+    size_t cand_half_off;  // u16 [N, H, list]: their fp16 maxima
+    size_t redo_off;       // int [N * H]: (row, head) pairs the rescoring kernel hands to the exact kernel
     size_t total;
     int max_items;
     int max_tiles;
+    int list;          // groups kept per row by the half-precision prefilter
+    bool tc;           // a tensor-core sweep runs (bf16 storage and a supported (d, k))
+    bool f16;          // ... namely the half-precision prefilter (score_select_f16.cu)
     bool reorder;      // the sweep runs the rows of large graphs in locality order (reorder.cu)
     bool prune;        // the sweep skips key tiles that cannot hold a candidate (prune.cu)
 };
 
 constexpr int64_t kReorderMinNodes = 32768;  // below this the extra launches cost more than they can save
 
-// `tc`: the tensor-core sweep will run (bf16 mode and a supported (d, k))
-inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, bool tc, bool prune = false) {
+bool score_select_tc_supported(int32_t d, int32_t k);
+bool score_select_f16_supported(int32_t d, int32_t k);
+int score_select_f16_list(int32_t k);
+
+// Which sweep the plan is for: the one the mode selects, or one a test entry point asks for.
+enum PlanVariant { kPlanByMode = 0, kPlanNoTensorCore = 1, kPlanTcFp32Acc = 2, kPlanTcFp16Acc = 3 };
+
+inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k, int mode,
+                                       int variant = kPlanByMode) {
     FwdWorkspace w;
     const int32_t g = G > 0 ? G : 1;
-    w.max_items = (int)(N / 128 + (G > 0 ? G : 1) + 1);
+    w.tc = variant == kPlanByMode ? (mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k))
+                                  : variant != kPlanNoTensorCore;
+    w.f16 = variant == kPlanByMode ? (w.tc && mode == KMIP_BF16_TC && score_select_f16_supported(d, k))
+                                   : variant == kPlanTcFp16Acc;
+    w.list = w.f16 ? score_select_f16_list(k) : 0;
+    w.max_items = (int)(N / 128 + g + 1);
     w.items_off = kStatusBytes;
     w.kpack_off = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
-    w.reorder = tc && N >= kReorderMinNodes;
-    w.qperm_off = align_up(w.kpack_off + (tc ? (size_t)N * H * d * 2 : 0));
-    w.perm_off = align_up(w.qperm_off + (w.reorder ? (size_t)N * H * d * 2 : 0));
+    w.reorder = w.tc && N >= kReorderMinNodes;
+    w.qperm_off = align_up(w.kpack_off + (w.tc ? (size_t)N * H * d * 2 : 0));
+    w.perm_off = align_up(w.qperm_off + ((w.reorder || w.f16) ? (size_t)N * H * d * 2 : 0));
     w.code_off = align_up(w.perm_off + (w.reorder ? (size_t)N * 4 : 0));
-    w.prune = prune && w.reorder;
+    w.prune = variant == kPlanByMode && mode == KMIP_BF16_TC_PRUNED && w.reorder;
     w.max_tiles = (int)(N / 128 + g + 2);  // tile0 of a graph = floor(first row / 128) + graph index
     const size_t p = w.prune ? 1 : 0, rec = (size_t)(d + 4) * 4;
     w.kperm_off = align_up(w.code_off + (w.reorder ? (size_t)N * 2 : 0));
@@ -86,7 +109,12 @@ inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t 
     w.qnorm_off = align_up(w.gmax_off + p * (size_t)g * 4);
     w.qstat_off = align_up(w.qnorm_off + p * (size_t)N * H * 4);
     w.kstat_off = align_up(w.qstat_off + p * (size_t)w.max_items * 3 * H * rec);
-    w.total = align_up(w.kstat_off + p * (size_t)w.max_tiles * H * rec);
+    const size_t f = w.f16 ? 1 : 0, rows = (size_t)N * H;
+    w.f16stat_off = align_up(w.kstat_off + p * (size_t)w.max_tiles * H * rec);
+    w.cand_word_off = align_up(w.f16stat_off + f * 16 * (size_t)H);
+    w.cand_half_off = align_up(w.cand_word_off + f * rows * w.list * 4);
+    w.redo_off = align_up(w.cand_half_off + f * rows * w.list * 2);
+    w.total = align_up(w.redo_off + f * rows * 4);
     return w;
 }
 
@@ -222,10 +250,17 @@ cudaError_t launch_score_select_exact(const FwdArgs& a);
 int sm_count();  // multiprocessors of the current device (cached per device)
 // score_select_tc.cu: tcgen05 scores + running top-k (bf16 storage); returns cudaErrorNotSupported
 // when (d, k) is outside what the tensor-core kernel covers
-bool score_select_tc_supported(int32_t d, int32_t k);
 int score_select_tc_rows_per_item(int32_t d, int32_t k);
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float* dump);
+// Half-precision prefilter of the tensor-core mode, head widths 16 and 32, k <= 32:
+// f16_convert.cu (norm maxima, scaled fp16 copies of K and Q), score_select_f16.cu (sweep: 384-row work items),
+// refine_f16.cu (exact rescoring, redo list), score_select_exact.cu (the listed rows again, from all keys)
+cudaError_t launch_f16_convert(const FwdArgs& a, const FwdWorkspace& w);
+cudaError_t launch_score_select_f16(const FwdArgs& a, const FwdWorkspace& w);
+cudaError_t launch_score_dump_f16(const FwdArgs& a, const FwdWorkspace& w, float* dump);
+cudaError_t launch_refine_f16(const FwdArgs& a, const FwdWorkspace& w);
+cudaError_t launch_score_select_exact_redo(const FwdArgs& a, const FwdWorkspace& w);
 // refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k
 cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_refine_topk_fp32(const FwdArgs& a);

@@ -385,6 +385,7 @@ cudaError_t launch_reorder_queries(const FwdArgs& a, const FwdWorkspace& w) {
         graph_sort_kernel<kCodeBits><<<std::min(n_graphs, sm_count() * 2), kSortThreads, (1 << kCodeBits) * 4, a.stream>>>(
             a.graph_offsets, a.G, (int)a.N, code, perm, sb);
     }
+    if (w.f16) return cudaGetLastError();  // the half-precision prefilter gathers while it converts (f16_convert.cu)
     const int vec_per_row = HD * 2 / 16;
     const long long n_vec = (long long)a.N * vec_per_row;
     gather_rows_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, a.stream>>>(

@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 score_select_exact_kernel(const T* __restrict__ Q, const T* __restrict__ K,
                           const int32_t* __restrict__ offs, int G, int N, int H, int k,
                           int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
-                          const StatusBlock* __restrict__ sb) {
+                          const StatusBlock* __restrict__ sb, const int* __restrict__ redo_list) {
     if (sb->status != KMIP_OK) return;  // the plan kernel rejected the offsets
     constexpr int CAP = 32 * E;
     constexpr int VEC = Elem<T>::kVec;
@@ -42,11 +42,13 @@ score_select_exact_kernel(const T* __restrict__ Q, const T* __restrict__ K,
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     cand_t* row = s_rows[wib];
     float* q = s_q[wib];
-    const long long n_rows = (long long)N * H;
+    // redo_list: only the (row, head) pairs the rescoring kernel of the half-precision prefilter listed
+    const long long n_rows = redo_list ? (long long)sb->n_redo : (long long)N * H;
     const int room = CAP - k;  // pending slots
 
-    for (long long r = (long long)blockIdx.x * kWarpsPerBlock + wib; r < n_rows;
-         r += (long long)gridDim.x * kWarpsPerBlock) {
+    for (long long x = (long long)blockIdx.x * kWarpsPerBlock + wib; x < n_rows;
+         x += (long long)gridDim.x * kWarpsPerBlock) {
+        const long long r = redo_list ? (long long)__ldg(redo_list + x) : x;
         const int i = (int)(r / H), h = (int)(r % H);
         int lo, hi;
         graph_range(offs, G, N, i, lo, hi);
@@ -89,9 +91,11 @@ score_select_exact_kernel(const T* __restrict__ Q, const T* __restrict__ K,
 }
 
 template <typename T, int D>
-cudaError_t launch_d(const FwdArgs& a) {
+cudaError_t launch_d(const FwdArgs& a, const int* redo_list = nullptr) {
     const long long n_rows = (long long)a.N * a.H;
-    const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 64);
+    // the redo pass does not know its row count on the host: a grid that covers a few thousand rows at once
+    const int blocks = redo_list ? sm_count() * 4
+                                 : (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 64);
     const T* Q = static_cast<const T*>(a.Q);
     const T* K = static_cast<const T*>(a.K);
     const dim3 grid(blocks), block(kWarpsPerBlock * 32);
@@ -99,7 +103,7 @@ cudaError_t launch_d(const FwdArgs& a) {
 #define KMIP_LAUNCH_EXACT(E_) \
     score_select_exact_kernel<T, D, E_><<<grid, block, 0, a.stream>>>( \
         Q, K, a.graph_offsets, a.G, (int)a.N, a.H, a.k, a.topk_idx, a.topk_score, \
-        reinterpret_cast<const StatusBlock*>(a.ws))
+        reinterpret_cast<const StatusBlock*>(a.ws), redo_list)
     if (a.k <= 16) KMIP_LAUNCH_EXACT(2);
     else if (a.k <= 96) KMIP_LAUNCH_EXACT(4);
     else KMIP_LAUNCH_EXACT(8);
@@ -122,6 +126,13 @@ cudaError_t launch_t(const FwdArgs& a) {
 
 cudaError_t launch_score_select_exact(const FwdArgs& a) {
     return a.mode == KMIP_FP32_EXACT ? launch_t<float>(a) : launch_t<__nv_bfloat16>(a);
+}
+
+// The rows the half-precision prefilter could not decide (bf16 storage, head widths 16 and 32), again
+// from all keys of their graph; overwrites their topk_idx / topk_score.
+cudaError_t launch_score_select_exact_redo(const FwdArgs& a, const FwdWorkspace& w) {
+    const int* redo = reinterpret_cast<const int*>(a.ws + w.redo_off);
+    return a.d == 16 ? launch_d<__nv_bfloat16, 16>(a, redo) : launch_d<__nv_bfloat16, 32>(a, redo);
 }
 
 }  // namespace kmip

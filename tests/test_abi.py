@@ -46,17 +46,26 @@ def test_version_and_status_strings(kb):
 def test_workspace_bytes_host_only(kb):
     f = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
     b = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
-    kq = 2 * 500_000 * 4 * 32 * 2                                           # bf16 copies of K (regrouped) and Q (sweep order)
-    assert kq < f < kq + 500_000 * 6 + (1 << 20)                           # + permutation, codes, work items
+    rows = 500_000 * 4
+    kq = 2 * rows * 32 * 2                                    # 2-byte copies of K (regrouped) and Q (sweep order)
+    lists = rows * (48 * 6 + 4)                               # half-precision prefilter: 48 groups of 6 bytes per row, redo list
+    assert kq + lists < f < kq + lists + 500_000 * 6 + (1 << 20)   # + permutation, codes, work items
+    assert f < 2 * rows * 32 * 2 * 4                          # linear in N*H*(d + k): nothing like N^2
     small = kb.kmip_attn_workspace_bytes(20_000, 1, 4, 32, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
-    assert 20_000 * 4 * 32 * 2 < small < 20_000 * 4 * 32 * 2 + (1 << 20)    # small problems keep their row order: K copy only
+    srows = 20_000 * 4
+    assert 2 * srows * 64 + srows * 292 < small < 2 * srows * 64 + srows * 292 + (1 << 20)
+    # d = 64 runs the fp32-accumulate sweep: one bf16 copy of K only while the row order is kept
+    wide = kb.kmip_attn_workspace_bytes(20_000, 1, 4, 64, 32, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
+    assert srows * 128 < wide < srows * 128 + (1 << 20)
     assert 256 < kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_FP32_EXACT, kb.PASS_FORWARD) < (1 << 20)
-    # pruned mode: 16 bytes per node + 4 per (node, head) + (d + 4) floats per (128 nodes, head) for the key tiles
-    # and three times that for the query tiles of the work items; the same as the plain mode below 32768 nodes
+    # pruned mode (fp32-accumulate sweep): copies of K and Q, 16 bytes per node + 4 per (node, head) + (d + 4)
+    # floats per (128 nodes, head) for the key tiles and three times that for the query tiles of the work
+    # items; below 32768 nodes it keeps the row order and needs the K copy only
     fp = kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_FORWARD)
     extra = 500_000 * (16 + 4 * 4) + 4 * (500_000 // 128 + 3) * 4 * 36 * 4
-    assert f + 500_000 * 16 < fp < f + extra + (1 << 16)
-    assert kb.kmip_attn_workspace_bytes(20_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_FORWARD) == small
+    assert kq + 500_000 * 16 < fp < kq + 500_000 * 6 + extra + (1 << 20)
+    sp = kb.kmip_attn_workspace_bytes(20_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_FORWARD)
+    assert srows * 64 < sp < srows * 64 + (1 << 20)
     assert kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_BACKWARD) == b
     pairs = 500_000 * 4 * 32
     assert 24 * pairs < b < 26 * pairs          # p, dS, 16-byte hit records: 24 bytes per selected pair + O(N*H)

@@ -274,5 +274,7 @@ def test_workspace_is_linear_in_n():
     a = kb.kmip_attn_workspace_bytes(100_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
     b = kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
     assert b < 10.5 * a and b < 1_000_000 * 4 * (6 * 16 + 4) * 4 + (1 << 20)   # 24 bytes per selected pair + per-row arrays
-    # forward: bf16 copies of K (regrouped) and Q (sweep order) + 6 bytes per node + work items
-    assert kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_FORWARD) < 2 * 1_000_000 * 4 * 32 * 2 + 8 * 1_000_000
+    # forward: 2-byte copies of K (regrouped) and Q (sweep order), the prefilter's 24 groups of 6 bytes and a redo
+    # slot per (node, head), 6 bytes per node, work items
+    rows = 1_000_000 * 4
+    assert kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_FORWARD) < 2 * rows * 32 * 2 + rows * (24 * 6 + 4) + 8 * 1_000_000
