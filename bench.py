@@ -29,6 +29,7 @@ METRIC = "k-MIP fwd+bwd query-key scores/sec at N=500k"
 UNIT = "scores/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 FWD_LAUNCHES = 5            # regroup keys, plan, score+select sweep, rescoring, softmax+gather-V
+F16_FWD_LAUNCHES = 8        # plan, norm maxima, K and Q conversions, prefilter sweep, rescoring, redo pass, softmax+gather-V
 REORDER_LAUNCHES = 3        # tensor-core mode from 32768 nodes on: locality codes, per-graph sort, permuted copy of Q
 BWD_LAUNCHES = 8            # rows, histogram, 3 scan kernels, fill, 2 segment kernels
 
@@ -160,7 +161,60 @@ def fwd_launches(w):
     tc = w.k <= 64 or (w.k <= 128 and w.d <= 64)
     if not tc:
         return 3
+    if w.d <= 32 and w.k <= 32:      # half-precision prefilter; the permuted copy of Q is made by its conversion kernel
+        return F16_FWD_LAUNCHES + (REORDER_LAUNCHES - 1 if w.N >= 32768 else 0)
     return FWD_LAUNCHES + (REORDER_LAUNCHES if w.N >= 32768 else 0)
+
+
+def sweep_kernel_name(w):
+    if w.mode != wl.MODE_BF16_TC:
+        return "score_select_fp32_kernel / score_select_exact_kernel (CUDA cores)"
+    if w.d <= 32 and w.k <= 32:
+        return "score_select_f16_kernel (tcgen05 fp16 prefilter scores + running top-(k+slack) of 8-key groups)"
+    return "score_select_tc_kernel (tcgen05 scores + running top-k of 8-key groups)"
+
+
+def measure_other_config(cfg, steps, peaks, dev):
+    """Forward + backward of another BASELINE config on the same GPU: per-stage times through the library's
+    profiling hooks, the sweep's fraction of the measured tensor peak.  Inputs resident, >= 3 warm-ups."""
+    import torch
+    from paper_2604_03815_b200 import binding as kb
+    w = wl.make_config(cfg)
+    dt = kb.storage_dtype(w.mode)
+    Q, K, V, dO = (torch.from_numpy(getattr(w, n)).to(dev, dt) for n in ("Q", "K", "V", "dOut"))
+    offs = torch.from_numpy(w.graph_offsets).to(dev)
+    fb = kb.ForwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode, dev)
+    bb = kb.BackwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode, dev)
+
+    def step():
+        rc = kb.kmip_attn_forward(Q, K, V, offs, w.k, w.mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace)
+        assert rc == kb.KMIP_OK, kb.status_string(rc)
+        rc = kb.kmip_attn_backward(Q, K, V, offs, w.k, w.mode, fb.out, dO, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK,
+                                   bb.dV, bb.workspace)
+        assert rc == kb.KMIP_OK, kb.status_string(rc)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
+    kb.kmip_profile_enable(steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    st, nf, nb = kb.kmip_profile_read()
+    kb.kmip_profile_enable(0)
+    sweep_ms = st["score_select"] / nf
+    fwd_ms = sum(st[s_] for s_ in kb.STAGES[:kb.N_FWD_STAGES]) / nf
+    tfl = 2.0 * w.d * w.n_scores / (sweep_ms * 1e-3) / 1e12
+    return {"workload": describe(w), "ms_per_step": e0.elapsed_time(e1) / steps, "fwd_ms": fwd_ms, "sweep_ms": sweep_ms,
+            "refine_ms": st["refine"] / nf, "bwd_ms": sum(st[s_] for s_ in kb.STAGES[kb.N_FWD_STAGES:]) / nb,
+            "value": float(w.n_scores) * steps / (e0.elapsed_time(e1) * 1e-3), "unit": UNIT,
+            "sweep_tflops": tfl, "frac": tfl / peaks["bf16_tflops"],
+            "fwd_frac": 2.0 * w.d * w.n_scores / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "redo_rows": kb.kmip_attn_sweep_counters(fb.workspace)[4]}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -317,6 +371,12 @@ def run_ours(args, w):
         }
         del fbp
 
+    # configs 3 and 5 of the benchmark's list, a few steps each (the headline stays config 4)
+    other = None
+    if args.config == 4 and not args.nodes and world == 1 and not args.no_other_configs:
+        peaks_o = load_peaks()
+        other = {f"c{c}": measure_other_config(c, 5, peaks_o, dev) for c in (3, 5)}
+
     e2e = e2e_setup()
     for _ in range(min(args.warmup, 2)):
         step_e2e()
@@ -347,12 +407,14 @@ def run_ours(args, w):
             traffic = tj.get("dram_bytes_per_launch")
     tensor_kernel = w.mode == wl.MODE_BF16_TC
     roofline = {
-        "kernel": "score_select_tc_kernel (tcgen05 scores + running top-k of 8-key groups)" if tensor_kernel else "score_select_exact_kernel",
+        "kernel": sweep_kernel_name(w),
         "bound": "tensor" if tensor_kernel else "alu",
         "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
         "frac": tflops / peaks["bf16_tflops"], "frac_of_sustained_peak": tflops / peaks["bf16_tflops_sustained"],
         "peak_source": f"{peaks['_source']} (burst cuBLAS bf16; sustained {peaks['bf16_tflops_sustained']})",
         "flops_per_launch": flops, "ms_per_launch": per_call["score_select"], "traffic": traffic,
+        "fwd_frac": flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"] if fwd_ms > 0 else None,
+        "fwd_frac_note": "the same flops over the whole forward pass (plan, conversions, sweep, rescoring, softmax+gather-V)",
     }
     pairs = w.N * w.H * w.k
     esz = 2 if w.mode == wl.MODE_BF16_TC else 4
@@ -376,17 +438,22 @@ def run_ours(args, w):
         "fwd_scores_per_s": w.n_scores / (fwd_ms * 1e-3) if fwd_ms > 0 else None,
         "rows_per_s": w.N * w.H / (1e-3 * (fwd_ms + bwd_ms)) if fwd_ms + bwd_ms > 0 else None,
         "hbm_stages": {
-            "softmax_gather_gbs": fwd_tail_bytes / (per_call["softmax_gather"] * 1e-3) / 1e9 if per_call["softmax_gather"] > 0 else None,
-            "backward_gbs": bwd_bytes / (bwd_ms * 1e-3) / 1e9 if bwd_ms > 0 else None,
+            "softmax_gather_algorithmic_gbs": fwd_tail_bytes / (per_call["softmax_gather"] * 1e-3) / 1e9 if per_call["softmax_gather"] > 0 else None,
+            "backward_algorithmic_gbs": bwd_bytes / (bwd_ms * 1e-3) / 1e9 if bwd_ms > 0 else None,
             "peak_gbs": peaks["hbm_gbs"],
+            "note": "algorithmic bytes over stage time: the gathered rows are served mostly from L2, so these are not DRAM "
+                    "rates; DRAM traffic per kernel (ncu) is in profiles/gather_backward_dram_config4_200k.md",
         },
         "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": 1e3 * secs_e2e / args.steps,
                 "overlap": "two device buffer sets: a step's copies overlap its neighbours' kernels, all inside the timed region",
+                "note": "copied back every step: out, dQ, dK, dV; topk_idx / topk_score (saved for the backward call) stay on the device",
                 "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host.values())),
                 "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for n, t in host_out.items()
                                               if w.backward or n == "out"))},
         "cuda_graph_replay_ms_per_step": graph_ms,
         "pruned": pruned,
+        "redo_rows": kb.kmip_attn_sweep_counters(fb.workspace)[4],
+        "other_configs": other,
         "gpu_launches": (fwd_launches(w) + (BWD_LAUNCHES if w.backward else 0)) * args.steps,
         "clocks": clocks,
     }
@@ -411,6 +478,7 @@ def main():
     ap.add_argument("--nodes", type=int, default=0, help="override the node count of configs 3/4 (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pruned", action="store_true", help="skip the extra measurement of the pruned mode")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the short runs of configs 3 and 5")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

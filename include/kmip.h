@@ -160,13 +160,15 @@ int kmip_attn_backward_dropout(const void *Q, const void *K, const void *V,
  * the share of the FULL softmax over all nodes of its graph that falls on the k keys kept by the
  * forward pass,
  *   mass[i,h] = sum_t exp(topk_score[i,h,t] / sqrt(d)) / sum_j exp(q_i^h . k_j^h / sqrt(d)),
- * a number in (0, 1]; 1 when the graph has at most k nodes.  Costs one more pass over all scores
- * (fp32 on CUDA cores), so it is meant for inspection, not for the training loop.
+ * a number in (0, 1]; 1 when the graph has at most k nodes.  It needs every score of the row once more.
+ * In the bf16 modes they come from the tensor cores (the pipeline of the forward sweep with a running
+ * log-sum-exp in place of the selection: about the cost of one forward sweep, every head width); in
+ * KMIP_FP32_EXACT mode they are fp32 sums on CUDA cores, about ten times slower, d = 128 not supported
+ * there (KMIP_ERR_UNSUPPORTED).  Meant for inspection, not for the training loop.
  * Inputs: Q, K, graph_offsets as for kmip_attn_forward; topk_score [N, H, k] as written by it.
  * Output (fully overwritten): mass, device memory, float [N, H], 4-byte aligned.
  * workspace: at least kmip_attn_workspace_bytes(..., KMIP_PASS_FORWARD) bytes; its contents are
  * overwritten, and its status block reports malformed offsets as for the forward pass.
- * d = 128 is not supported here (KMIP_ERR_UNSUPPORTED).
  */
 int kmip_attn_topk_mass(const void *Q, const void *K,
                         const int32_t *graph_offsets, int32_t G, int64_t N,

@@ -138,3 +138,63 @@ def topk_mass(Q, K, graph_offsets, k, rows=None):
     if rc != 0:
         raise ValueError(f"kmip_oracle_topk_mass failed with status {rc}")
     return mass
+
+
+# ------------------------------------------------------------------------------------------------
+# The full layer of Eq. 2 / Algorithm 1 ("Require" line and lines 2-8): projections in front of the
+# attention core and the output projection behind it.  Plain numpy matrix products in fp64 around the
+# C functions above; the selection is the oracle's own top-k or an index set supplied by the caller.
+# ------------------------------------------------------------------------------------------------
+def _round_bf16(a):
+    """Round fp64/fp32 values to the nearest bfloat16 (ties to even), returned as float64."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    out = (r & 0xFFFFFFFF).astype(np.uint32).view(np.float32).astype(np.float64)
+    return np.where(np.isfinite(f), out, f.astype(np.float64))
+
+
+def _store(a, storage):
+    """What the attention core receives: its inputs are stored as bf16 or fp32 arrays."""
+    if storage == "bf16":
+        return _round_bf16(a)
+    return np.ascontiguousarray(a, dtype=np.float32).astype(np.float64)
+
+
+def layer_forward(x, w_q, w_k, w_v, w_o, graph_offsets, H, k, idx=None, storage="f32"):
+    """Y = sum_h O^h W_O^h with O^h = kMIP-Attn(X W_Q^h, X W_K^h, X W_V^h) per graph (Eq. 2).
+
+    x [N, d_model]; w_q, w_k, w_v [H*d, d_model] (row h*d + c is column c of W^h); w_o [d_model, H*d].
+    Q, K, V and O pass through `storage` ("bf16" or "f32": the arrays the core reads and writes).
+    idx: index set [N, H, k] to use instead of the oracle's own top-k (Algorithm 1 line 3).
+    Returns dict(y, q, k, v, o, idx) with fp64 arrays."""
+    x = np.asarray(x, dtype=np.float64)
+    N = x.shape[0]
+    d = w_q.shape[0] // H
+    q = _store(x @ np.asarray(w_q, np.float64).T, storage).reshape(N, H, d)
+    kk = _store(x @ np.asarray(w_k, np.float64).T, storage).reshape(N, H, d)
+    v = _store(x @ np.asarray(w_v, np.float64).T, storage).reshape(N, H, d)
+    if idx is None:
+        f = forward(q, kk, v, graph_offsets, k)
+        o, idx = f["out"], f["idx"]
+    else:
+        o, _ = forward_given_idx(q, kk, v, idx)
+    o = _store(o, storage)
+    y = o.reshape(N, H * d) @ np.asarray(w_o, np.float64).T
+    return {"y": y, "q": q, "k": kk, "v": v, "o": o, "idx": np.asarray(idx, dtype=np.int32)}
+
+
+def layer_backward(x, w_q, w_k, w_v, w_o, H, fwd, d_y):
+    """Gradients of sum(y * d_y) through layer_forward with the selection fwd["idx"] held constant (Sec. 3.1)
+    and the storage roundings treated as the identity; returns dict(dx, dw_q, dw_k, dw_v, dw_o) in fp64."""
+    x = np.asarray(x, dtype=np.float64)
+    d_y = np.asarray(d_y, dtype=np.float64)
+    N = x.shape[0]
+    d = w_q.shape[0] // H
+    o_cat = fwd["o"].reshape(N, H * d)
+    dw_o = d_y.T @ o_cat
+    d_o = (d_y @ np.asarray(w_o, np.float64)).reshape(N, H, d)
+    dq, dk, dv = backward(fwd["q"], fwd["k"], fwd["v"], d_o, fwd["idx"])
+    dq, dk, dv = (g.reshape(N, H * d) for g in (dq, dk, dv))
+    dx = dq @ np.asarray(w_q, np.float64) + dk @ np.asarray(w_k, np.float64) + dv @ np.asarray(w_v, np.float64)
+    return {"dx": dx, "dw_q": dq.T @ x, "dw_k": dk.T @ x, "dw_v": dv.T @ x, "dw_o": dw_o}

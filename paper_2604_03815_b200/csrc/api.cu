@@ -128,7 +128,9 @@ int forward_impl(const void* Q, const void* K, const void* V, const int32_t* gra
     // about twice, below that the one-warp-per-row kernel has more parallelism
     const bool tiled32 = mode == KMIP_FP32_EXACT && score_select_fp32_tiled_supported(d, k) &&
                          (a.fp32_path == 0 ? (N / 128) * H >= 2 * sm_count() : a.fp32_path == 2);
-    if (launch_plan(a, w, tc ? score_select_tc_rows_per_item(d, k) : 128) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_plan(a, w, w.f16 ? score_select_f16_rows_per_item(k) : tc ? score_select_tc_rows_per_item(d, k) : 128) !=
+        cudaSuccess)
+        return KMIP_ERR_CUDA;
     if (w.reorder && launch_reorder_queries(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.f16 && launch_f16_convert(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.prune && (launch_reorder_keys(a, w) != cudaSuccess || launch_prune_stats(a, w) != cudaSuccess)) return KMIP_ERR_CUDA;
@@ -191,18 +193,26 @@ int kmip_attn_topk_mass(const void* Q, const void* K, const int32_t* graph_offse
                         size_t workspace_bytes, void* stream) {
     const int rc = check_shape(N, H, d, k, mode);
     if (rc != KMIP_OK) return rc;
-    if (d > 64) return KMIP_ERR_UNSUPPORTED;
+    const bool tensor = mode != KMIP_FP32_EXACT;  // bf16 storage: the scores come from the tensor cores
+    if (!tensor && d > 64) return KMIP_ERR_UNSUPPORTED;
     if (N == 0) return KMIP_OK;
     if (graph_offsets != nullptr && G < 1) return KMIP_ERR_INVALID_ARG;
     if (!Q || !K || !topk_score || !mass || !workspace) return KMIP_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(topk_score) || !aligned16(workspace) ||
         (reinterpret_cast<uintptr_t>(mass) & 3u) || (reinterpret_cast<uintptr_t>(graph_offsets) & 3u))
         return KMIP_ERR_INVALID_ARG;
-    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, k, mode, kPlanNoTensorCore);
+    const FwdWorkspace w = plan_fwd_workspace(N, graph_offsets ? G : 1, H, d, k, mode,
+                                              tensor ? kPlanTcFp32AccInOrder : kPlanNoTensorCore);
     if (workspace_bytes < w.total) return KMIP_ERR_WORKSPACE;
     FwdArgs a{Q, K, nullptr, graph_offsets, graph_offsets ? G : 1, N, H, d, k, mode, nullptr, nullptr,
               const_cast<float*>(topk_score), static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (tensor) {
+        if (launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
+        if (launch_plan(a, w, score_select_tc_rows_per_item(d, 1)) != cudaSuccess) return KMIP_ERR_CUDA;
+        if (launch_topk_mass_tc(a, w, mass) != cudaSuccess) return KMIP_ERR_CUDA;
+        return KMIP_OK;
+    }
     if (launch_plan(a, w, 128) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_topk_mass(a, w, mass) != cudaSuccess) return KMIP_ERR_CUDA;
     return KMIP_OK;
@@ -280,7 +290,7 @@ int kmip_test_sweep_order(const void* workspace, int64_t N, int32_t G, int32_t H
     if (rc != KMIP_OK) return rc;
     if (!workspace || !order || !rows_per_item || G < 0) return KMIP_ERR_INVALID_ARG;
     const FwdWorkspace w = plan_fwd_workspace(N, G > 0 ? G : 1, H, d, k, mode);
-    *rows_per_item = w.tc ? score_select_tc_rows_per_item(d, k) : 128;
+    *rows_per_item = w.f16 ? score_select_f16_rows_per_item(k) : w.tc ? score_select_tc_rows_per_item(d, k) : 128;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (w.reorder) {
         if (cudaMemcpy(order, static_cast<const unsigned char*>(workspace) + w.perm_off, (size_t)N * 4,
@@ -320,7 +330,7 @@ int kmip_test_f16_scores(const void* Q, const void* K, int64_t N, int32_t H, int
     FwdArgs a{Q, K, nullptr, nullptr, 1, N, H, d, 1, KMIP_BF16_TC, nullptr, nullptr, nullptr,
               static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream)};
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
-    if (launch_plan(a, w, score_select_tc_rows_per_item(d, 1)) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_plan(a, w, score_select_f16_rows_per_item(1)) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_f16_convert(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
     if (launch_score_dump_f16(a, w, scores) != cudaSuccess) return KMIP_ERR_CUDA;
     // per head: {q_n2max, k_n2max, k_first16_n2max, 0} as the conversion measured them

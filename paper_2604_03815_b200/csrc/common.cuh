@@ -78,9 +78,12 @@ constexpr int64_t kReorderMinNodes = 32768;  // below this the extra launches co
 bool score_select_tc_supported(int32_t d, int32_t k);
 bool score_select_f16_supported(int32_t d, int32_t k);
 int score_select_f16_list(int32_t k);
+int score_select_f16_rows_per_item(int32_t k);
+int score_select_f16x4_rows_per_item();
 
 // Which sweep the plan is for: the one the mode selects, or one a test entry point asks for.
-enum PlanVariant { kPlanByMode = 0, kPlanNoTensorCore = 1, kPlanTcFp32Acc = 2, kPlanTcFp16Acc = 3 };
+enum PlanVariant { kPlanByMode = 0, kPlanNoTensorCore = 1, kPlanTcFp32Acc = 2, kPlanTcFp16Acc = 3,
+                   kPlanTcFp32AccInOrder = 4 /* fp32-accumulate sweep over the rows in their own order */ };
 
 inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k, int mode,
                                        int variant = kPlanByMode) {
@@ -94,7 +97,7 @@ inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t 
     w.max_items = (int)(N / 128 + g + 1);
     w.items_off = kStatusBytes;
     w.kpack_off = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
-    w.reorder = w.tc && N >= kReorderMinNodes;
+    w.reorder = w.tc && N >= kReorderMinNodes && variant != kPlanTcFp32AccInOrder;
     w.qperm_off = align_up(w.kpack_off + (w.tc ? (size_t)N * H * d * 2 : 0));
     w.perm_off = align_up(w.qperm_off + ((w.reorder || w.f16) ? (size_t)N * H * d * 2 : 0));
     w.code_off = align_up(w.perm_off + (w.reorder ? (size_t)N * 4 : 0));
@@ -258,14 +261,17 @@ cudaError_t launch_score_dump_tc(const FwdArgs& a, const FwdWorkspace& w, float*
 // refine_f16.cu (exact rescoring, redo list), score_select_exact.cu (the listed rows again, from all keys)
 cudaError_t launch_f16_convert(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_select_f16(const FwdArgs& a, const FwdWorkspace& w);
+cudaError_t launch_score_select_f16x4(const FwdArgs& a, const FwdWorkspace& w);  // k <= 16, called by the above
 cudaError_t launch_score_dump_f16(const FwdArgs& a, const FwdWorkspace& w, float* dump);
 cudaError_t launch_refine_f16(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_score_select_exact_redo(const FwdArgs& a, const FwdWorkspace& w);
 // refine.cu: rescoring of the k best 8-key groups left by the tensor-core sweep -> final top-k
 cudaError_t launch_refine_topk(const FwdArgs& a, const FwdWorkspace& w);
 cudaError_t launch_refine_topk_fp32(const FwdArgs& a);
-// topk_mass.cu: share of the full softmax held by the kept scores; needs 128-row work items in the workspace
+// topk_mass.cu: share of the full softmax held by the kept scores on CUDA cores (fp32 storage); needs 128-row
+// work items in the workspace.  score_select_tc.cu: the same on the tensor cores (bf16 storage, every head width)
 cudaError_t launch_topk_mass(const FwdArgs& a, const FwdWorkspace& w, float* mass);
+cudaError_t launch_topk_mass_tc(const FwdArgs& a, const FwdWorkspace& w, float* mass);
 // tiled CUDA-core sweep of fp32 mode (score_select_fp32.cu): 128-row work items, then launch_refine_topk_fp32
 bool score_select_fp32_tiled_supported(int32_t d, int32_t k);
 cudaError_t launch_score_select_fp32_tiled(const FwdArgs& a, const FwdWorkspace& w);

@@ -300,6 +300,13 @@ __device__ __forceinline__ uint32_t warp_ballot_half_gt(uint32_t m, uint32_t t) 
     return r;
 }
 
+// 2^x on the special-function unit (about 2 ulp; -inf gives 0)
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // max of three floats in one instruction (sm_100+)
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;

@@ -76,13 +76,19 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int t = e * 32 + lane;
-            word[e] = 0xFFFFFFFFu;
+            word[e] = 0u;
             g[e] = -CUDART_INF_F;
+            valid[e] = false;
             if (t < LIST) {
-                word[e] = __ldg(cand_word + (size_t)r * LIST + t);
-                g[e] = __half2float(__ushort_as_half(__ldg(cand_half + (size_t)r * LIST + t)));
+                const unsigned short hb = __ldg(cand_half + (size_t)r * LIST + t);
+                // empty slots: the four-pipeline sweep marks them by the half 0xFFFF and never writes their
+                // group word, the ring sweep writes an all-ones word
+                if (hb != 0xFFFFu) {
+                    word[e] = __ldg(cand_word + (size_t)r * LIST + t);
+                    valid[e] = word[e] != 0xFFFFFFFFu;
+                    if (valid[e]) g[e] = __half2float(__ushort_as_half(hb));
+                }
             }
-            valid[e] = word[e] != 0xFFFFFFFFu;
             n_valid += __popc(__ballot_sync(FULL, valid[e]));
         }
 

@@ -1,5 +1,5 @@
 // Half-precision prefilter sweep of the tensor-core mode (Algorithm 1 lines 2-3) for head widths
-// 16 and 32 and k <= 32.
+// 16 and 32 and 16 < k <= 32 (k <= 16: score_select_f16x4.cu, the same filter on another pipeline).
 //
 // The paper lists half-precision arithmetic and tensor-core support as the engineering it left open
 // (Sec. 6; closing remark of the FlashAttention comparison in the appendix).  The sweep of
@@ -574,9 +574,7 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
 
 template <int D, bool DUMP>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
-    // (list blocks, query tiles per CTA, key stages, pending slots per row) by k; shared memory decides
-    if (a.k <= 8) return launch_cfg<D, 2, 3, 4, 24, DUMP>(a, w, dump);
-    if (a.k <= 16) return launch_cfg<D, 3, 3, 4, 24, DUMP>(a, w, dump);
+    // (list blocks, query tiles per CTA, key stages, pending slots per row); shared memory decides
     return launch_cfg<D, 6, 3, 3, 22, DUMP>(a, w, dump);
 }
 
@@ -584,14 +582,12 @@ cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
 
 bool score_select_f16_supported(int32_t d, int32_t k) { return (d == 16 || d == 32) && k <= 32; }
 int score_select_f16_list(int32_t k) { return k <= 8 ? 16 : k <= 16 ? 24 : 48; }
+// lists of up to 24 groups (k <= 16) run the four-pipeline kernel of score_select_f16x4.cu with 512-row work items
+int score_select_f16_rows_per_item(int32_t k) { return k <= 16 ? score_select_f16x4_rows_per_item() : 3 * BM; }
 
 cudaError_t launch_score_select_f16(const FwdArgs& a, const FwdWorkspace& w) {
+    if (a.k <= 16) return launch_score_select_f16x4(a, w);
     return a.d == 16 ? launch_d<16, false>(a, w, nullptr) : launch_d<32, false>(a, w, nullptr);
-}
-
-// Test entry: the fp16 scores themselves (scaled as the converted operands are), dump[h][i][j], ld = N.
-cudaError_t launch_score_dump_f16(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
-    return a.d == 16 ? launch_d<16, true>(a, w, dump) : launch_d<32, true>(a, w, dump);
 }
 
 }  // namespace kmip

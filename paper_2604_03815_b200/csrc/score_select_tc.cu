@@ -271,14 +271,18 @@ __device__ __forceinline__ void publish_thresholds(float tau, float inv_qn, int 
     }
 }
 
-template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE>
+// LSE: instead of selecting, the selection warps fold every score of a row into a running log-sum-exp
+// (base 2, scale log2(e)/sqrt(d)) and write the share of the full softmax that the row's k kept scores
+// hold - the cumulative-attention-weight diagnostic of the paper's appendix "Additional results" - to
+// `dump` as float [N, H]; `topk_score` is then an input.
+template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE, bool LSE = false>
 __global__ void __launch_bounds__(NQT * 128 + 96, 1)
 score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const WorkItem* __restrict__ items, StatusBlock* __restrict__ sb, int H, int k,
                        int32_t* __restrict__ topk_idx, float* __restrict__ topk_score,
                        float* __restrict__ dump, int dump_ld /* = N */, long long wait_limit, int drop_first_tile,
                        const int* __restrict__ perm, const PruneArgs pr) {
-    static_assert(!(DUMP && PRUNE), "the score dump sweeps every tile");
+    static_assert(!(DUMP && PRUNE) && !(LSE && (DUMP || PRUNE)), "the score dump and the softmax-share pass sweep every tile");
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
     constexpr int NEPI = 4 * NQT;
@@ -344,7 +348,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // rest idle.  Those units are cut into their 128-row query tiles instead, one CTA each - a CTA with a
     // single busy warp group gets through its key tiles faster - provided the pieces fit one wave.
     long long n_whole = total, n_units = total;
-    if (!PRUNE && !DUMP && NQT > 1 && total > (long long)gridDim.x) {
+    if (!PRUNE && !DUMP && !LSE && NQT > 1 && total > (long long)gridDim.x) {
         const long long left = total % gridDim.x;
         if (left * NQT <= (long long)gridDim.x) { n_whole = total - left; n_units = n_whole + left * NQT; }
     }
@@ -705,6 +709,64 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         break;
                     }
                 }
+            } else if constexpr (LSE) {
+                // running maximum and sum of 2^(c (s - m)) over all keys of the graph, 64 columns at a time
+                const float c2 = 1.4426950408889634f * rsqrtf((float)D);
+                float m_run = -CUDART_INF_F, l_run = 0.0f;
+                for (int j = 0; j < ntiles; ++j, ++tcnt) {
+                    const int b = (tcnt * NQT + qt) & (NBUF - 1);
+                    ok = wait_or_abort(full_bar0 + (uint32_t)b * (8u * NQT), (uint32_t)(tcnt >> kUseShift) & 1u, sAbort, sb,
+                                       6, wait_limit);
+                    ok = __all_sync(FULL, ok);
+                    if (!ok) break;
+                    if (quarter == 0 && lane == 0) ptx::mbar_arrive(bars.k_empty(tcnt % S));
+                    ptx::tc_fence_after();
+                    const uint32_t taddr = taddr0 + (uint32_t)(b * BN);
+                    const int ncol = it.key_hi - (it.key_lo + j * BN);  // columns that exist; below 128 only in the last tile
+#pragma unroll 1
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t v[64];
+                        ptx::tmem_ld_32x64_sync(taddr + half * 64, v);
+                        if (half == 1) {
+                            ptx::tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bars.t_empty(b));
+                        }
+                        if (ncol < BN) {
+#pragma unroll
+                            for (int x = 0; x < 64; ++x)
+                                if (half * 64 + x >= ncol) v[x] = 0xFF800000u;  // -inf
+                        }
+                        float hm[8];
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const int o = 8 * g;
+                            const float a0 = ptx::max3(__uint_as_float(v[o]), __uint_as_float(v[o + 1]), __uint_as_float(v[o + 2]));
+                            const float a1 = ptx::max3(__uint_as_float(v[o + 3]), __uint_as_float(v[o + 4]), __uint_as_float(v[o + 5]));
+                            hm[g] = ptx::max3(a0, a1, fmaxf(__uint_as_float(v[o + 6]), __uint_as_float(v[o + 7])));
+                        }
+                        const float tm = fmaxf(ptx::max3(hm[0], hm[1], hm[2]), ptx::max3(hm[3], hm[4], ptx::max3(hm[5], hm[6], hm[7])));
+                        const float m_new = fmaxf(m_run, tm);
+                        if (m_new > -CUDART_INF_F) {  // false only while every column so far was past the key range
+                            const float off = -m_new * c2;
+                            float add[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                            for (int x = 0; x < 64; ++x) add[x & 3] += ptx::ex2(fmaf(__uint_as_float(v[x]), c2, off));
+                            l_run = l_run * ptx::ex2(fmaf(m_run, c2, off)) + ((add[0] + add[1]) + (add[2] + add[3]));
+                            m_run = m_new;
+                        }
+                    }
+                }
+                if (ok && rvalid) {
+                    const size_t o = (size_t)(it.row0 + local) * H + h;
+                    const float* sc = topk_score + o * k;
+                    float top = 0.0f;
+                    for (int t = 0; t < k; ++t) {
+                        const float x = __ldg(sc + t);
+                        if (x > -CUDART_INF_F) top += ptx::ex2((x - m_run) * c2);
+                    }
+                    dump[o] = l_run > 0.0f ? fminf(top / l_run, 1.0f) : 0.0f;
+                }
             } else {
                 const int ragged_j = ((it.key_hi - it.key_lo) & (BN - 1)) ? ntiles - 1 : -1;  // only the last tile can be short
                 int key0 = it.key_lo;
@@ -775,7 +837,7 @@ score_select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 }
             }
             if (!ok) break;
-            if (!DUMP && active) {
+            if (!DUMP && !LSE && active) {
                 // finalise: drain the pending slots, then store each row's k groups (first key and
                 // group maximum, unsorted; empty slots as -1 / -inf) for the rescoring kernel
                 flush_pending<KG>(rs, wl_s, wp_addr, rvalid);
@@ -840,7 +902,7 @@ bool make_tensor_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t ro
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE>
+template <int D, int KG, int NQT, int S, bool DUMP, bool PRUNE, bool LSE = false>
 cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     using Sh = TcShape<D>;
     using Sp = SmemPlan<KG, NQT, S>;
@@ -851,7 +913,7 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     if (!make_tensor_map<D>(&tmQ, w.reorder ? static_cast<const void*>(a.ws + w.qperm_off) : a.Q, a.N, (int64_t)a.H * D) ||
         !make_tensor_map<D>(&tmK, a.ws + w.kpack_off, a.N * a.H, D))
         return cudaErrorInvalidValue;
-    auto kern = score_select_tc_kernel<D, KG, NQT, S, DUMP, PRUNE>;
+    auto kern = score_select_tc_kernel<D, KG, NQT, S, DUMP, PRUNE, LSE>;
     PruneArgs pr{nullptr, nullptr, nullptr};
     if (PRUNE)
         pr = PruneArgs{reinterpret_cast<const float*>(a.ws + w.qstat_off), reinterpret_cast<const float*>(a.ws + w.kstat_off),
@@ -922,6 +984,18 @@ int score_select_tc_rows_per_item(int32_t d, int32_t k) {  // 128 * query tiles 
 
 cudaError_t launch_score_select_tc(const FwdArgs& a, const FwdWorkspace& w) {
     return w.prune ? launch_any<false, true>(a, w, nullptr) : launch_any<false, false>(a, w, nullptr);
+}
+
+// The softmax-share diagnostic on the tensor cores: mass[i,h] as float [N, H].  The workspace must hold the
+// regrouped keys and work items of score_select_tc_rows_per_item(d, 1) rows; the rows keep their order.
+cudaError_t launch_topk_mass_tc(const FwdArgs& a, const FwdWorkspace& w, float* mass) {
+    switch (a.d) {
+        case 16: return launch_cfg<16, 4, 3, 4, false, false, true>(a, w, mass);
+        case 32: return launch_cfg<32, 4, 3, 4, false, false, true>(a, w, mass);
+        case 64: return launch_cfg<64, 4, 2, 3, false, false, true>(a, w, mass);
+        case 128: return launch_cfg<128, 4, 1, 3, false, false, true>(a, w, mass);
+        default: return cudaErrorNotSupported;
+    }
 }
 
 // Test hook: same TMA / tcgen05 pipeline, but the selection warps write every score of the tile to

@@ -47,8 +47,8 @@ def stratified_rows(w, fb, n, seed=2468):
     by the structure of the data, not only by row number:
       * borders of work items and of their 128-row query tiles in SWEEP order (the sweep runs the rows of
         large graphs in a data-dependent locality order), for the first, last and a few middle items;
-      * every row of up to four work items of the schedule's tail, whose units the sweep cuts into single
-        query tiles with one CTA each (a different code path from the body of the schedule);
+      * every row of up to four work items of the schedule's tail (the units past the last full wave of
+        CTAs, which the sweep may cut into single query tiles with one CTA each: a different code path);
       * every cluster of the point-cloud workload and hub / non-hub rows of every graph of the hub batch;
       * the row-number strata of workloads.sample_rows (graph borders, block borders) and seeded uniform picks.
     Returns sorted unique int64 row numbers."""
@@ -68,7 +68,8 @@ def stratified_rows(w, fb, n, seed=2468):
     n_sms = torch.cuda.get_device_properties(0).multi_processor_count
     total, nqt = n_items * w.H, rpi // 128
     left = total % n_sms if total > n_sms else 0
-    tail = sorted({u % n_items for u in range(total - left, total)}) if (nqt > 1 and left and left * nqt <= n_sms) else []
+    # (cut into single query tiles with one CTA each when the pieces fit one wave, otherwise a last partial wave)
+    tail = sorted({u % n_items for u in range(total - left, total)}) if (nqt > 1 and left) else []
     for it in (tail[:2] + tail[-2:]) if len(tail) > 4 else tail:
         r0, nr = items[it]
         picks.append(order[r0:r0 + nr])

@@ -44,7 +44,7 @@ def test_config3_100k_nodes():
 def test_config4_500k_point_cloud():
     st = _full(4, 4096)
     assert st["identical_rows"] > 0.95
-    assert st["tail_items"] >= 4        # the sample holds whole work items of the schedule's split tail
+    assert st["tail_items"] >= 4        # the sample holds whole work items of the schedule's tail
 
 
 def test_config5_hub_batch():

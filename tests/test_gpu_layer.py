@@ -1,8 +1,6 @@
-"""The full attention layer (Eq. 2: projections, k-MIP attention core, output projection) against an
-fp64 PyTorch restatement on the CPU: same bf16-rounded weights and inputs, the selection the GPU made
-is checked against dense fp64 scores and then held fixed, as the paper's backward pass holds it."""
-import math
-
+"""The full attention layer (Eq. 2: projections, k-MIP attention core, output projection) against the
+CPU oracle's layer functions: same bf16-rounded weights and inputs, the selection the GPU made is checked
+against the oracle's dense fp64 scores and then held fixed, as the paper's backward pass holds it."""
 import numpy as np
 import pytest
 import torch
@@ -10,37 +8,18 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-def _bf16_st(t):
-    """Round to bf16 with a straight-through gradient (the GPU stores Q, K, V and O in bf16)."""
-    return t + (t.to(torch.bfloat16).to(t.dtype) - t).detach()
-
-
-def _reference(x, wq, wk, wv, wo, idx, H, d, rounding):
-    N = x.shape[0]
-    r = _bf16_st if rounding else (lambda t: t)
-    q = r(x @ wq.T).view(N, H, d)
-    k = r(x @ wk.T).view(N, H, d)
-    v = r(x @ wv.T).view(N, H, d)
-    safe = idx.clamp(min=0).long()                                  # [N, H, k]
-    hh = torch.arange(H)[None, :, None].expand_as(safe)
-    ks, vs = k[safe, hh], v[safe, hh]                               # [N, H, k, d]
-    s = (q[:, :, None, :] * ks).sum(-1) / math.sqrt(d)
-    s = s.masked_fill(idx < 0, float("-inf"))
-    p = torch.softmax(s, dim=-1)
-    o = r((p[..., None] * vs).sum(2))
-    return r(o.reshape(N, H * d) @ wo.T), q, k
-
-
 @pytest.mark.parametrize("dtype,d_head,k", [(torch.bfloat16, 16, 8), (torch.bfloat16, 32, 16), (torch.float32, 32, 5),
                                             (torch.float32, 10, 10), (torch.bfloat16, 40, 6)])
 def test_layer_forward_and_gradients(dtype, d_head, k):
+    from oracle import kmip_oracle as oracle
     from paper_2604_03815_b200.layer import KMIPSelfAttention
 
     torch.manual_seed(1234)
     d_model, H = 64, 4
     sizes = [200, 1, 300, 37]
     N = sum(sizes)
-    offs = torch.tensor(np.concatenate([[0], np.cumsum(sizes)]), dtype=torch.int32, device="cuda")
+    offs_np = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    offs = torch.tensor(offs_np, dtype=torch.int32, device="cuda")
     layer = KMIPSelfAttention(d_model, H, d_head, k, dtype=dtype)
     x = torch.randn(N, d_model, device="cuda").to(dtype).requires_grad_(True)
     g = torch.randn(N, d_model, device="cuda").to(dtype)
@@ -48,40 +27,38 @@ def test_layer_forward_and_gradients(dtype, d_head, k):
     (y.float() * g.float()).sum().backward()
     torch.cuda.synchronize()
 
-    # fp64 restatement with the same (rounded) parameters
-    x64 = x.detach().double().cpu().requires_grad_(True)
-    ws = [p.detach().double().cpu().requires_grad_(True) for p in (layer.w_q.weight, layer.w_k.weight, layer.w_v.weight, layer.w_o.weight)]
-    idx_c = idx.cpu()
-    y64, q64, k64 = _reference(x64, *ws, idx_c, H, d_head, rounding=dtype == torch.bfloat16)
-    (y64 * g.double().cpu()).sum().backward()
+    # the oracle's layer on the same (rounded) parameters, with the GPU's selection
+    f64 = lambda t: t.detach().double().cpu().numpy()
+    xs, ws = f64(x), [f64(p) for p in (layer.w_q.weight, layer.w_k.weight, layer.w_v.weight, layer.w_o.weight)]
+    storage = "bf16" if dtype == torch.bfloat16 else "f32"
+    idx_np = idx.cpu().numpy()
+    fwd = oracle.layer_forward(xs, *ws, offs_np, H, k, idx=idx_np, storage=storage)
+    grads = oracle.layer_backward(xs, *ws, H, fwd, f64(g))
 
     # the selection: inside the query's graph, no duplicates, and no selected key worse than the
-    # k-th best dense fp64 score by more than 1e-2 relative
-    o = offs.cpu().numpy().astype(np.int64)
-    qn, kn, idn = q64.detach().numpy(), k64.detach().numpy(), idx_c.numpy()
-    for gi in range(len(sizes)):
-        lo, hi = o[gi], o[gi + 1]
-        if hi == lo:
-            continue
-        keff = min(k, hi - lo)
-        for h in range(H):
-            S = qn[lo:hi, h] @ kn[lo:hi, h].T
-            kth = np.sort(S, axis=1)[:, ::-1][:, keff - 1]
-            sel = idn[lo:hi, h, :keff]
-            assert np.all((sel >= lo) & (sel < hi)) and np.all(idn[lo:hi, h, keff:] == -1)
-            assert all(len(set(r)) == keff for r in sel.tolist())
-            ssel = np.take_along_axis(S, sel - lo, axis=1)
-            assert np.all(ssel.min(axis=1) >= kth - 1e-2 * np.abs(kth))
+    # k-th best dense fp64 score (of the oracle's own Q and K) by more than 1e-2 relative
+    own = oracle.forward(fwd["q"], fwd["k"], fwd["v"], offs_np, k)
+    _, exact = oracle.forward_given_idx(fwd["q"], fwd["k"], fwd["v"], idx_np)
+    gi = np.searchsorted(offs_np, np.arange(N), side="right") - 1
+    lo, hi = offs_np[gi].astype(np.int64), offs_np[gi + 1].astype(np.int64)
+    keff = np.minimum(k, hi - lo)
+    valid = np.arange(k)[None, None, :] < keff[:, None, None]
+    assert np.all(((idx_np >= lo[:, None, None]) & (idx_np < hi[:, None, None])) | ~valid) and np.all((idx_np == -1) | valid)
+    srt = np.sort(np.where(valid, idx_np, -1 - np.arange(k)[None, None, :]), axis=-1)
+    assert np.all(np.diff(srt, axis=-1) != 0)
+    kth = np.take_along_axis(own["score"], np.maximum(keff - 1, 0)[:, None, None].repeat(H, 1), axis=2)[..., 0]
+    worst = np.where(valid, exact, np.inf).min(axis=-1)
+    assert np.all(worst >= kth - 1e-2 * np.abs(kth))
 
     def close(a, b, what):
-        a, b = a.double().cpu(), b.double()
-        tol = (3e-2 if dtype == torch.bfloat16 else 2e-4) * max(1.0, float(b.abs().max()))
-        assert float((a - b).abs().max()) <= tol, f"{what}: {float((a - b).abs().max()):.3e} > {tol:.3e}"
+        a = a.detach().double().cpu().numpy()
+        tol = (3e-2 if dtype == torch.bfloat16 else 2e-4) * max(1.0, float(np.abs(b).max()))
+        assert float(np.abs(a - b).max()) <= tol, f"{what}: {float(np.abs(a - b).max()):.3e} > {tol:.3e}"
 
-    close(y.detach(), y64.detach(), "output")
-    close(x.grad, x64.grad, "d/dx")
-    for p, w64, name in zip((layer.w_q.weight, layer.w_k.weight, layer.w_v.weight, layer.w_o.weight), ws, "QKVO"):
-        close(p.grad, w64.grad, f"d/dW_{name}")
+    close(y, fwd["y"], "output")
+    close(x.grad, grads["dx"], "d/dx")
+    for p, name in zip((layer.w_q.weight, layer.w_k.weight, layer.w_v.weight, layer.w_o.weight), "qkvo"):
+        close(p.grad, grads["dw_" + name], f"d/dW_{name}")
 
 
 def test_layer_attention_dropout_only_in_training():

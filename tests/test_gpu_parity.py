@@ -95,10 +95,10 @@ def test_ragged_batch_with_tiny_and_empty_graphs(mode):
 
 
 def test_item_and_ring_boundaries():
-    """Graphs around the 384-row work-item size of the d <= 32, k <= 32 sweep: one, two or three
-    active query tiles, a short last key tile, and enough key tiles per item for the ring of
-    accumulator buffers and its barrier phases to wrap several times."""
-    sizes = [383, 384, 385, 769, 1153, 2000, 127, 128, 129]
+    """Graphs around the 512-row and 384-row work-item sizes of the sweeps: one to four active query
+    tiles, a short last key tile, and enough key tiles per item for the accumulator buffers and their
+    barrier phases to wrap several times."""
+    sizes = [383, 384, 385, 511, 512, 513, 769, 1025, 1153, 2000, 127, 128, 129]
     for d, k in ((32, 32), (16, 16)):
         w = wl.iid_workload("s", 90 + d, sizes, 2, d, k, wl.MODE_BF16_TC, input_scale=1.0 / np.sqrt(d))
         st = _fwd_bwd(w)

@@ -15,6 +15,7 @@ if torch.cuda.is_available():
 
 
 @pytest.mark.parametrize("mode,d,k,scale", [(wl.MODE_BF16_TC, 32, 16, 1.0), (wl.MODE_BF16_TC, 16, 5, 0.25),
+                                            (wl.MODE_BF16_TC, 64, 40, 0.5), (wl.MODE_BF16_TC, 128, 7, 0.3),
                                             (wl.MODE_FP32_EXACT, 64, 8, 0.5)])
 def test_topk_mass_matches_the_oracle(mode, d, k, scale):
     sizes = [700, 3, 0, 129, 64, 1]
@@ -35,8 +36,22 @@ def test_topk_mass_matches_the_oracle(mode, d, k, scale):
     assert ref.min() < 0.9                                                   # and the case is not trivial
 
 
+def test_topk_mass_on_a_graph_of_many_tiles_with_clusters():
+    """Clustered queries and keys (peaked softmax, large scores) over a graph that spans dozens of key tiles
+    and several work items, with a ragged last tile; the tensor-core pass against the oracle."""
+    w = wl.make_config(4, N=5003, H=2, d=32, k=32)
+    Q, K, V, dO, offs = pu.to_device(w)
+    fb = kb.forward(Q, K, V, offs, w.k, w.mode)
+    mass = torch.full((w.N, w.H), -1.0, dtype=torch.float32, device="cuda")
+    assert kb.kmip_attn_topk_mass(Q, K, offs, w.k, w.mode, fb.topk_score, mass, fb.workspace) == kb.KMIP_OK
+    assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK
+    got = mass.cpu().numpy().astype(np.float64)
+    ref = oracle.topk_mass(w.Q, w.K, w.graph_offsets, w.k)
+    np.testing.assert_allclose(got, ref, rtol=2e-3, atol=1e-6)
+
+
 def test_topk_mass_argument_checks():
-    w = wl.iid_workload("s", 5100, [64], 1, 128, 4, wl.MODE_BF16_TC)
+    w = wl.iid_workload("s", 5100, [64], 1, 128, 4, wl.MODE_FP32_EXACT)
     Q, K, V, dO, offs = pu.to_device(w)
     fb = kb.forward(Q, K, V, offs, 4, w.mode)
     mass = torch.zeros((w.N, 1), dtype=torch.float32, device="cuda")

@@ -441,3 +441,72 @@ def test_bad_arguments_are_rejected():
         oracle.forward(Q, K, V, np.array([0, 4], dtype=np.int32), 2)         # does not end at N
     with pytest.raises(ValueError):
         oracle.forward(Q, K, V, None, 2, rows=np.array([9], dtype=np.int64))
+
+
+# ------------------------------------------------------------------ the full layer (Eq. 2, Algorithm 1 lines 2-8)
+def _layer_case(seed, N=40, d_model=12, H=3, d=4):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((N, d_model))
+    ws = [rng.standard_normal((H * d, d_model)) / np.sqrt(d_model) for _ in range(3)]
+    w_o = rng.standard_normal((d_model, H * d)) / np.sqrt(H * d)
+    return x, ws[0], ws[1], ws[2], w_o
+
+
+def test_layer_with_k_equal_n_is_multi_head_attention():
+    """Eq. 2 with T_k keeping everything is textbook multi-head self-attention inside each graph:
+    independent check with torch's own linear and scaled_dot_product_attention in fp64."""
+    import torch
+    x, wq, wk, wv, wo = _layer_case(1)
+    N, H, d = x.shape[0], 3, 4
+    offs = np.array([0, 25, 40], dtype=np.int32)
+    got = oracle.layer_forward(x, wq, wk, wv, wo, offs, H, 25)["y"]
+    xt = torch.from_numpy(x)
+    lin = lambda w: torch.nn.functional.linear(xt, torch.from_numpy(w)).view(N, H, d).transpose(0, 1)   # [H, N, d]
+    q, k, v = lin(wq), lin(wk), lin(wv)
+    o = torch.zeros(H, N, d, dtype=torch.float64)
+    for lo, hi in ((0, 25), (25, 40)):
+        o[:, lo:hi] = torch.nn.functional.scaled_dot_product_attention(q[:, lo:hi], k[:, lo:hi], v[:, lo:hi])
+    ref = torch.nn.functional.linear(o.transpose(0, 1).reshape(N, H * d), torch.from_numpy(wo)).numpy()
+    np.testing.assert_allclose(got, ref, rtol=0, atol=2e-6)      # Q, K, V, O pass through fp32 storage in the oracle
+
+
+def test_layer_with_identity_projections_is_the_core():
+    rng = np.random.default_rng(2)
+    N, H, d = 30, 2, 4
+    x = rng.standard_normal((N, H * d)).astype(np.float32).astype(np.float64)
+    eye = np.eye(H * d)
+    f = oracle.layer_forward(x, eye, eye, eye, eye, None, H, 5)
+    core = oracle.forward(x.reshape(N, H, d), x.reshape(N, H, d), x.reshape(N, H, d), None, 5)
+    assert np.array_equal(f["idx"], core["idx"])
+    np.testing.assert_allclose(f["y"], core["out"].reshape(N, H * d), rtol=0, atol=1e-6)
+
+
+def test_layer_backward_matches_central_differences_with_frozen_selection():
+    x, wq, wk, wv, wo = _layer_case(3, N=24)
+    H, k = 3, 4
+    offs = np.array([0, 14, 24], dtype=np.int32)
+    rng = np.random.default_rng(4)
+    dy = rng.standard_normal((x.shape[0], wo.shape[0]))
+    fwd = oracle.layer_forward(x, wq, wk, wv, wo, offs, H, k)
+    g = oracle.layer_backward(x, wq, wk, wv, wo, H, fwd, dy)
+    loss = lambda *a: float((oracle.layer_forward(*a, offs, H, k, idx=fwd["idx"])["y"] * dy).sum())
+    args = [x, wq, wk, wv, wo]
+    eps = 2e-3
+    for pos, name in enumerate(("dx", "dw_q", "dw_k", "dw_v", "dw_o")):
+        for _ in range(6):
+            i, j = rng.integers(0, args[pos].shape[0]), rng.integers(0, args[pos].shape[1])
+            hi_, lo_ = [a.copy() for a in args], [a.copy() for a in args]
+            hi_[pos][i, j] += eps
+            lo_[pos][i, j] -= eps
+            fd = (loss(*hi_) - loss(*lo_)) / (2 * eps)
+            assert abs(fd - g[name][i, j]) <= 2e-3 * max(1.0, abs(fd)), (name, i, j, fd, g[name][i, j])
+
+
+def test_layer_bf16_storage_rounds_what_the_core_reads():
+    x, wq, wk, wv, wo = _layer_case(5)
+    f = oracle.layer_forward(x, wq, wk, wv, wo, None, 3, 6, storage="bf16")
+    for name in ("q", "k", "v", "o"):
+        a = f[name].astype(np.float32)
+        assert np.array_equal(a.view(np.uint32) & 0xFFFF, np.zeros_like(a, dtype=np.uint32))   # bf16-representable
+    exact = x @ wq.T
+    assert np.max(np.abs(f["q"].reshape(exact.shape) - exact)) <= 2.0 ** -8 * np.max(np.abs(exact))
