@@ -47,7 +47,9 @@ typedef enum {
     KMIP_ERR_CUDA = 4,         /* a CUDA runtime call or a kernel launch failed */
     KMIP_ERR_TIMEOUT = 5,      /* device side: a bounded wait inside a kernel ran out */
     KMIP_ERR_BAD_OFFSETS = 6,  /* device side: graph_offsets is not a valid CSR row-pointer array */
-    KMIP_ERR_TOO_LARGE = 7     /* kmip_attn_forward_static_scratch: the problem needs more than the built-in scratch */
+    KMIP_ERR_TOO_LARGE = 7,    /* kmip_attn_forward_static_scratch: the problem needs more than the built-in scratch */
+    KMIP_ERR_CHECK = 8         /* device side, only in a library built with -DKMIP_CHECKS: an index test failed or a
+                                  canary block between two workspace regions was overwritten */
 } kmip_status_t;
 
 typedef enum {
@@ -252,6 +254,14 @@ const char *kmip_status_string(int status);
 
 /* Library version, major*10000 + minor*100 + patch. */
 int kmip_version(void);
+
+/*
+ * Build flags of the loaded library: bit 0 is set in a -DKMIP_CHECKS build (libkmip_checks.so), which puts
+ * 256-byte canary blocks between the regions of every workspace (kmip_attn_workspace_bytes of that library
+ * already counts them), verifies them after each pass and tests indices before following them; problems
+ * are reported as KMIP_ERR_CHECK in the status word, never by a trap.  Slower; for debugging and tests.
+ */
+int kmip_build_flags(void);
 
 #ifdef __cplusplus
 }

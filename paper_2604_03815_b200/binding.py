@@ -25,7 +25,10 @@ KMIP_BF16_TC_PRUNED = 2
 PASS_FORWARD = 0
 PASS_BACKWARD = 1
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libkmip.so")
+# KMIP_LIBRARY selects another build of the same library, e.g. libkmip_checks.so (canary blocks and device-side
+# index tests, see kmip_build_flags in include/kmip.h)
+LIB_PATH = os.environ.get("KMIP_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libkmip.so")
+KMIP_ERR_CHECK = 8
 _lib = None
 
 
@@ -51,6 +54,7 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(LIB_PATH)
         P, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
         L.kmip_version.restype = ctypes.c_int
+        L.kmip_build_flags.restype = ctypes.c_int
         L.kmip_status_string.restype = ctypes.c_char_p
         L.kmip_status_string.argtypes = [ctypes.c_int]
         L.kmip_attn_workspace_bytes.restype = ctypes.c_int
@@ -95,6 +99,11 @@ def lib() -> ctypes.CDLL:
 
 def kmip_version() -> int:
     return int(lib().kmip_version())
+
+
+def kmip_build_flags() -> int:
+    """Bit 0: the loaded library is a -DKMIP_CHECKS build."""
+    return int(lib().kmip_build_flags())
 
 
 def status_string(status: int) -> str:

@@ -11,6 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libkmip.so")
+LIB_CHECKS = os.path.join(HERE, "libkmip_checks.so")   # the same sources with -DKMIP_CHECKS (see include/kmip.h, kmip_build_flags)
 SOURCES = ["api.cu", "plan.cu", "reorder.cu", "prune.cu", "score_select_exact.cu", "score_select_fp32.cu", "score_select_tc.cu", "score_select_f16.cu", "score_select_f16x4.cu", "f16_convert.cu", "refine.cu", "refine_f16.cu", "epilogue.cu", "backward.cu", "topk_mass.cu",
            "static_scratch.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -23,17 +24,19 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu for sm_100a and link libkmip.so; skipped when up to date."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
-        return LIB
-    os.makedirs(OBJ, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, checks: bool = False) -> str:
+    """Compile every .cu for sm_100a and link libkmip.so (checks=True: libkmip_checks.so, the build with
+    canary blocks and device-side index tests); skipped when up to date."""
+    lib, obj_dir = (LIB_CHECKS, OBJ + "_checks") if checks else (LIB, OBJ)
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _deps_mtime():
+        return lib
+    os.makedirs(obj_dir, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
-    if os.environ.get("KMIP_SWEEP_DEBUG") == "1":   # timing experiments of the sweep kernel (developer builds)
-        extra.append("-DKMIP_SWEEP_DEBUG=1")
+    if checks:
+        extra.append("-DKMIP_CHECKS")
 
     def compile_one(src):
-        obj = os.path.join(OBJ, src.replace(".cu", ".o"))
+        obj = os.path.join(obj_dir, src.replace(".cu", ".o"))
         cmd = [NVCC, *FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
@@ -44,14 +47,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(compile_one, SOURCES))
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     r = subprocess.run([NVCC, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"],
                        capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checks="--checks" in sys.argv))

@@ -39,7 +39,9 @@ int forward_impl(const void* Q, const void* K, const void* V, const int32_t* gra
 
 extern "C" {
 
-int kmip_version(void) { return 100; }
+int kmip_version(void) { return 200; }
+
+int kmip_build_flags(void) { return kChecks ? 1 : 0; }
 
 const char* kmip_status_string(int status) {
     switch (status) {
@@ -51,6 +53,7 @@ const char* kmip_status_string(int status) {
         case KMIP_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case KMIP_ERR_BAD_OFFSETS: return "graph_offsets is not a valid CSR offset array";
         case KMIP_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in array holds";
+        case KMIP_ERR_CHECK: return "a device-side index test or workspace canary of a KMIP_CHECKS build failed";
         default: return "unknown status";
     }
 }
@@ -121,6 +124,7 @@ int forward_impl(const void* Q, const void* K, const void* V, const int32_t* gra
         a.fp32_path = opt->fp32_path;
     }
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_canary_fill(a.ws, w.canaries, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_fwd < g_prof.max_calls) ? g_prof.fwd[g_prof.n_fwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
     if (tc && !w.prune && !w.f16 && launch_pack_keys(a, w) != cudaSuccess) return KMIP_ERR_CUDA;
@@ -146,6 +150,7 @@ int forward_impl(const void* Q, const void* K, const void* V, const int32_t* gra
     if (ev) cudaEventRecord(ev[3], a.stream);
     if (launch_softmax_gather(a) != cudaSuccess) return KMIP_ERR_CUDA;
     if (ev) cudaEventRecord(ev[4], a.stream);
+    if (launch_canary_check(a.ws, w.canaries, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     return KMIP_OK;
 }
 
@@ -182,9 +187,11 @@ int kmip_attn_backward_dropout(const void* Q, const void* K, const void* V, cons
     a.drop_p = drop_p;
     a.seed = seed;
     if (cudaMemsetAsync(a.ws, 0, kStatusBytes, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_canary_fill(a.ws, w.canaries, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     cudaEvent_t* ev = (g_prof.on && g_prof.n_bwd < g_prof.max_calls) ? g_prof.bwd[g_prof.n_bwd++] : nullptr;
     if (ev) cudaEventRecord(ev[0], a.stream);
     if (launch_backward(a, w, ev ? ev + 1 : nullptr) != cudaSuccess) return KMIP_ERR_CUDA;
+    if (launch_canary_check(a.ws, w.canaries, a.stream) != cudaSuccess) return KMIP_ERR_CUDA;
     return KMIP_OK;
 }
 

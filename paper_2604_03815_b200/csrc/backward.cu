@@ -88,10 +88,11 @@ bwd_rows_kernel(const T* __restrict__ K, const T* __restrict__ V, const T* __res
 
 // --------------------------------------------------------------------------------------- inverse
 __global__ void hist_kernel(const int32_t* __restrict__ topk_idx, long long n_pairs, int N, int H, int k,
-                            int* __restrict__ counts) {
+                            int* __restrict__ counts, StatusBlock* __restrict__ sb) {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_pairs) return;
     const int j = __ldg(topk_idx + e);
+    kmip_check(j < N, sb, 105);  // checks builds: an index the forward pass cannot have written (ignored either way)
     if (j < 0 || j >= N) return;
     const int h = (int)((e / k) % H);
     atomicAdd(counts + (size_t)j * H + h, 1);
@@ -210,7 +211,8 @@ scan_write_kernel(int* __restrict__ counts, long long n, const int* __restrict__
 // score gradient dS - instead of a pair id that would cost two more scattered 4-byte reads per hit.
 __global__ void fill_kernel(const int32_t* __restrict__ topk_idx, long long n_pairs, int N, int H, int k,
                             const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
-                            const int* __restrict__ seg_off, int* __restrict__ cursor, int4* __restrict__ hits) {
+                            const int* __restrict__ seg_off, int* __restrict__ cursor, int4* __restrict__ hits,
+                            StatusBlock* __restrict__ sb) {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_pairs) return;
     const int j = __ldg(topk_idx + e);
@@ -218,7 +220,9 @@ __global__ void fill_kernel(const int32_t* __restrict__ topk_idx, long long n_pa
     const long long r = e / k;  // query * H + head
     const int h = (int)(r % H);
     const size_t key = (size_t)j * H + h;
-    hits[seg_off[key] + atomicAdd(cursor + key, 1)] =
+    const long long pos = (long long)seg_off[key] + atomicAdd(cursor + key, 1);
+    if (!kmip_check(pos >= 0 && pos < n_pairs, sb, 104)) return;  // checks builds: inside the hit lists
+    hits[pos] =
         make_int4((int)(r / H), __float_as_int(__ldg(ws_p + e)), __float_as_int(__ldg(ws_ds + e)), 0);
 }
 
@@ -392,12 +396,12 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     if (ev) cudaEventRecord(ev[0], a.stream);
 
     const int pair_blocks = (int)((n_pairs + 255) / 256);
-    hist_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, cursor);
+    hist_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, cursor, sb);
     scan_block_sums_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums);
     scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(block_sums, w.scan_blocks);
     scan_write_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums, seg_off, long_list, sb);
     fill_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, ws_p, ws_ds, seg_off, cursor,
-                                                  hits);
+                                                  hits, sb);
     if (ev) cudaEventRecord(ev[1], a.stream);
 
     bwd_segments_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(

@@ -16,6 +16,25 @@ namespace kmip {
 constexpr size_t kStatusBytes = 256;
 constexpr size_t kAlign = 256;
 
+// -DKMIP_CHECKS builds (libkmip_checks.so) stand in for a memory checker: every workspace region is
+// preceded by a 256-byte canary block that a tail kernel verifies, and the kernels test the indices they
+// are about to follow.  A failed test RECORDS KMIP_ERR_CHECK in the status word and skips the access;
+// nothing traps.  Release builds compile all of it away.
+#ifdef KMIP_CHECKS
+constexpr bool kChecks = true;
+#else
+constexpr bool kChecks = false;
+#endif
+constexpr size_t kCanaryBytes = kChecks ? 256 : 0;
+constexpr uint32_t kCanaryWord = 0xC0DEFACEu;
+constexpr int kMaxCanaries = 24;
+
+// Offsets of the canary blocks of a workspace (checks builds; n = 0 otherwise).
+struct Canaries {
+    size_t off[kMaxCanaries];
+    int n = 0;
+};
+
 struct StatusBlock {
     int status;      // kmip_status_t recorded by the device (first error wins)
     int detail;      // where it happened (kernel-specific code)
@@ -71,6 +90,7 @@ struct FwdWorkspace {
     bool f16;          // ... namely the half-precision prefilter (score_select_f16.cu)
     bool reorder;      // the sweep runs the rows of large graphs in locality order (reorder.cu)
     bool prune;        // the sweep skips key tiles that cannot hold a candidate (prune.cu)
+    Canaries canaries;
 };
 
 constexpr int64_t kReorderMinNodes = 32768;  // below this the extra launches cost more than they can save
@@ -88,6 +108,12 @@ enum PlanVariant { kPlanByMode = 0, kPlanNoTensorCore = 1, kPlanTcFp32Acc = 2, k
 inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k, int mode,
                                        int variant = kPlanByMode) {
     FwdWorkspace w;
+    // start of the next region after one that ends at `end`; checks builds put a canary block in front of it
+    auto region = [&w](size_t end) {
+        const size_t c = align_up(end);
+        if (kChecks && w.canaries.n < kMaxCanaries) w.canaries.off[w.canaries.n++] = c;
+        return c + kCanaryBytes;
+    };
     const int32_t g = G > 0 ? G : 1;
     w.tc = variant == kPlanByMode ? (mode != KMIP_FP32_EXACT && score_select_tc_supported(d, k))
                                   : variant != kPlanNoTensorCore;
@@ -95,29 +121,29 @@ inline FwdWorkspace plan_fwd_workspace(int64_t N, int32_t G, int32_t H, int32_t 
                                    : variant == kPlanTcFp16Acc;
     w.list = w.f16 ? score_select_f16_list(k) : 0;
     w.max_items = (int)(N / 128 + g + 1);
-    w.items_off = kStatusBytes;
-    w.kpack_off = align_up(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
+    w.items_off = region(kStatusBytes);
+    w.kpack_off = region(w.items_off + sizeof(WorkItem) * (size_t)w.max_items);
     w.reorder = w.tc && N >= kReorderMinNodes && variant != kPlanTcFp32AccInOrder;
-    w.qperm_off = align_up(w.kpack_off + (w.tc ? (size_t)N * H * d * 2 : 0));
-    w.perm_off = align_up(w.qperm_off + ((w.reorder || w.f16) ? (size_t)N * H * d * 2 : 0));
-    w.code_off = align_up(w.perm_off + (w.reorder ? (size_t)N * 4 : 0));
+    w.qperm_off = region(w.kpack_off + (w.tc ? (size_t)N * H * d * 2 : 0));
+    w.perm_off = region(w.qperm_off + ((w.reorder || w.f16) ? (size_t)N * H * d * 2 : 0));
+    w.code_off = region(w.perm_off + (w.reorder ? (size_t)N * 4 : 0));
     w.prune = variant == kPlanByMode && mode == KMIP_BF16_TC_PRUNED && w.reorder;
     w.max_tiles = (int)(N / 128 + g + 2);  // tile0 of a graph = floor(first row / 128) + graph index
     const size_t p = w.prune ? 1 : 0, rec = (size_t)(d + 4) * 4;
-    w.kperm_off = align_up(w.code_off + (w.reorder ? (size_t)N * 2 : 0));
-    w.kcode_off = align_up(w.kperm_off + p * (size_t)N * 4);
-    w.kcs_off = align_up(w.kcode_off + p * (size_t)N * 2);
-    w.knorm_off = align_up(w.kcs_off + p * (size_t)N * 2);
-    w.gmax_off = align_up(w.knorm_off + p * (size_t)N * 4);
-    w.qnorm_off = align_up(w.gmax_off + p * (size_t)g * 4);
-    w.qstat_off = align_up(w.qnorm_off + p * (size_t)N * H * 4);
-    w.kstat_off = align_up(w.qstat_off + p * (size_t)w.max_items * 3 * H * rec);
+    w.kperm_off = region(w.code_off + (w.reorder ? (size_t)N * 2 : 0));
+    w.kcode_off = region(w.kperm_off + p * (size_t)N * 4);
+    w.kcs_off = region(w.kcode_off + p * (size_t)N * 2);
+    w.knorm_off = region(w.kcs_off + p * (size_t)N * 2);
+    w.gmax_off = region(w.knorm_off + p * (size_t)N * 4);
+    w.qnorm_off = region(w.gmax_off + p * (size_t)g * 4);
+    w.qstat_off = region(w.qnorm_off + p * (size_t)N * H * 4);
+    w.kstat_off = region(w.qstat_off + p * (size_t)w.max_items * 3 * H * rec);
     const size_t f = w.f16 ? 1 : 0, rows = (size_t)N * H;
-    w.f16stat_off = align_up(w.kstat_off + p * (size_t)w.max_tiles * H * rec);
-    w.cand_word_off = align_up(w.f16stat_off + f * 16 * (size_t)H);
-    w.cand_half_off = align_up(w.cand_word_off + f * rows * w.list * 4);
-    w.redo_off = align_up(w.cand_half_off + f * rows * w.list * 2);
-    w.total = align_up(w.redo_off + f * rows * 4);
+    w.f16stat_off = region(w.kstat_off + p * (size_t)w.max_tiles * H * rec);
+    w.cand_word_off = region(w.f16stat_off + f * 16 * (size_t)H);
+    w.cand_half_off = region(w.cand_word_off + f * rows * w.list * 4);
+    w.redo_off = region(w.cand_half_off + f * rows * w.list * 2);
+    w.total = region(w.redo_off + f * rows * 4);  // checks builds: a last canary block behind the last region
     return w;
 }
 
@@ -131,6 +157,7 @@ struct BwdWorkspace {
     size_t long_off;      // int   [N*H]     ids of long segments
     size_t total;
     int scan_blocks;
+    Canaries canaries;
 };
 
 constexpr int kScanItemsPerBlock = 4096;
@@ -139,14 +166,19 @@ inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
     BwdWorkspace w;
     const size_t rows = (size_t)N * H, pairs = rows * (size_t)k;
     w.scan_blocks = (int)((rows + 1 + kScanItemsPerBlock - 1) / kScanItemsPerBlock);
-    size_t o = kStatusBytes;
-    w.p_off = o;        o = align_up(o + 4 * pairs);
-    w.ds_off = o;       o = align_up(o + 4 * pairs);
-    w.seg_off = o;      o = align_up(o + 4 * (rows + 1));
-    w.cursor_off = o;   o = align_up(o + 4 * (rows + 1));
-    w.pairs_off = o;    o = align_up(o + 16 * pairs);
-    w.blocksum_off = o; o = align_up(o + 4 * (size_t)(w.scan_blocks + 1));
-    w.long_off = o;     o = align_up(o + 4 * rows);
+    auto region = [&w](size_t end) {
+        const size_t c = align_up(end);
+        if (kChecks && w.canaries.n < kMaxCanaries) w.canaries.off[w.canaries.n++] = c;
+        return c + kCanaryBytes;
+    };
+    size_t o = region(kStatusBytes);
+    w.p_off = o;        o = region(o + 4 * pairs);
+    w.ds_off = o;       o = region(o + 4 * pairs);
+    w.seg_off = o;      o = region(o + 4 * (rows + 1));
+    w.cursor_off = o;   o = region(o + 4 * (rows + 1));
+    w.pairs_off = o;    o = region(o + 16 * pairs);
+    w.blocksum_off = o; o = region(o + 4 * (size_t)(w.scan_blocks + 1));
+    w.long_off = o;     o = region(o + 4 * rows);
     w.total = o;
     return w;
 }
@@ -156,6 +188,13 @@ inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
 // ---------------------------------------------------------------------------------------------
 __device__ inline void record_status(StatusBlock* sb, int status, int detail) {
     if (atomicCAS(&sb->status, 0, status) == 0) sb->detail = detail;
+}
+// Checks builds: `cond` must hold before an index is followed; if it does not, the failure is recorded with
+// `code` (which test, see the call sites) and the caller skips the access.  Release builds: always true, no code.
+__device__ __forceinline__ bool kmip_check(bool cond, StatusBlock* sb, int code) {
+    if (!kChecks) return true;
+    if (!cond) record_status(sb, KMIP_ERR_CHECK, code);
+    return cond;
 }
 
 template <typename T> struct Elem;
@@ -236,6 +275,9 @@ struct BwdArgs {
     unsigned long long seed = 0ull;
 };
 
+// plan.cu, checks builds: write the canary blocks of a workspace / verify them (detail = 900 + block number)
+cudaError_t launch_canary_fill(unsigned char* ws, const Canaries& c, cudaStream_t stream);
+cudaError_t launch_canary_check(unsigned char* ws, const Canaries& c, cudaStream_t stream);
 // plan.cu: validates the offsets and writes the work items of the tensor-core kernel
 cudaError_t launch_plan(const FwdArgs& a, const FwdWorkspace& w, int rows_per_item);
 // plan.cu: K [N, H, d] -> [H, N, d] so that a head's key tile is one contiguous block for TMA

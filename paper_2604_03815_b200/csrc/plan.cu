@@ -92,7 +92,30 @@ __global__ void pack_keys_kernel(const uint4* __restrict__ K, uint4* __restrict_
     Kp[((long long)h * N + j) * vec_per_row + c] = __ldg(K + v);
 }
 
+__global__ void canary_kernel(unsigned char* __restrict__ ws, const Canaries c, bool fill) {
+    const int blk = blockIdx.x;
+    if (blk >= c.n) return;
+    uint32_t* p = reinterpret_cast<uint32_t*>(ws + c.off[blk]);
+    StatusBlock* sb = reinterpret_cast<StatusBlock*>(ws);
+    for (int i = threadIdx.x; i < (int)(kCanaryBytes / 4); i += blockDim.x) {
+        if (fill) p[i] = kCanaryWord;
+        else if (p[i] != kCanaryWord) record_status(sb, KMIP_ERR_CHECK, 900 + blk);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_canary_fill(unsigned char* ws, const Canaries& c, cudaStream_t stream) {
+    if (!kChecks || c.n == 0) return cudaSuccess;
+    canary_kernel<<<c.n, 64, 0, stream>>>(ws, c, true);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_canary_check(unsigned char* ws, const Canaries& c, cudaStream_t stream) {
+    if (!kChecks || c.n == 0) return cudaSuccess;
+    canary_kernel<<<c.n, 64, 0, stream>>>(ws, c, false);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_pack_keys(const FwdArgs& a, const FwdWorkspace& w) {
     const int vec_per_row = a.d * 2 / 16;

@@ -75,7 +75,14 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
         for (int t = lane; t < k; t += 32) row[t] = 0ull;
         __syncwarp();
 
-        float tau = floor_tau;
+        // Two attempts at most.  The margin above is relative to theta, so when the k-th best group maximum
+        // lies within rounding of zero the fp32 sums below can fall short of it by more than the margin and a
+        // key of the answer would be dropped; the row then comes out with fewer than k keys although its
+        // groups hold more, and it is scanned again without a floor.
+        for (int attempt = 0; attempt < 2; ++attempt) {
+        const float floor_now = attempt == 0 ? floor_tau : -CUDART_INF_F;
+        int n_seen = 0;  // keys of the row's groups that exist (inside the graph)
+        float tau = floor_now;
         int cnt = 0;
         constexpr int GPR = 32 / kGroup;           // groups scored per step (one key per lane)
         constexpr int NV = D * (int)sizeof(T) / 16;  // 16-byte vectors per key row
@@ -92,7 +99,8 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                 for (int e = 0; e < 4; ++e)
                     if (e == (tb >> 5)) g = __shfl_sync(0xFFFFFFFFu, gid[e], t & 31);
                 jj[u] = g + (lane % kGroup);
-                valid[u] = t < k && g >= 0 && jj[u] < hi;
+                valid[u] = t < k && g >= 0 && jj[u] < hi &&
+                           kmip_check(jj[u] >= 0 && hi <= N, const_cast<StatusBlock*>(sb), 101);  // checks builds: key row inside K
                 if (valid[u]) {
                     // regrouped by head, the 8 keys of a group are 8 consecutive rows
                     const uint4* kr = reinterpret_cast<const uint4*>(
@@ -119,6 +127,7 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                         }
                     }
                 }
+                n_seen += __popc(__ballot_sync(0xFFFFFFFFu, valid[u]));
                 const bool pass = valid[u] && (s > tau);
                 const unsigned m = __ballot_sync(0xFFFFFFFFu, pass);
                 if (m) {
@@ -126,7 +135,7 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
                     if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, kperm ? __ldg(kperm + jj[u]) : jj[u]);
                     cnt += __popc(m);
                     if (cnt > room - 32) {
-                        tau = fmaxf(floor_tau, E <= 4 ? warp_merge_row_chunks(row, k, cnt, lane) : warp_compact_row<E>(row, k, cnt, lane));
+                        tau = fmaxf(floor_now, E <= 4 ? warp_merge_row_chunks(row, k, cnt, lane) : warp_compact_row<E>(row, k, cnt, lane));
                         cnt = 0;
                     }
                 }
@@ -134,6 +143,16 @@ refine_topk_kernel(const T* __restrict__ Q, const T* __restrict__ Kp, const int3
         }
         // E <= 4 serves k <= 32: one kept key per lane, so the pending keys can be merged in 32-key chunks
         if (E <= 4) warp_merge_row_chunks(row, k, cnt, lane); else warp_compact_row<E>(row, k, cnt, lane);
+        __syncwarp();
+        const int n_kept = __popc(__ballot_sync(0xFFFFFFFFu, lane < k && row[lane] != 0ull)) +
+                           ((k > 32) ? __popc(__ballot_sync(0xFFFFFFFFu, lane + 32 < k && row[lane + 32] != 0ull)) +
+                                       __popc(__ballot_sync(0xFFFFFFFFu, lane + 64 < k && row[lane + 64] != 0ull)) +
+                                       __popc(__ballot_sync(0xFFFFFFFFu, lane + 96 < k && row[lane + 96] != 0ull)) : 0);
+        if (n_kept >= min(k, n_seen)) break;
+        __syncwarp();
+        for (int t = lane; t < k; t += 32) row[t] = 0ull;
+        __syncwarp();
+        }
         warp_store_row(row, k, lane, topk_idx + (size_t)r * k, topk_score + (size_t)r * k);
     }
 }

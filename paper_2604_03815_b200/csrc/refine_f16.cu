@@ -171,7 +171,7 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
                 const int t = t0 + u * 4 + (lane >> 3);
                 const uint32_t wd = t < n_kept ? words[t] : 0u;
                 jj[u] = (int)(wd & 0x7FFFFFFFu) + (int)(wd >> 31) + 2 * (lane & 7);
-                kv[u] = t < n_kept && jj[u] < hi;
+                kv[u] = t < n_kept && jj[u] < hi && kmip_check(jj[u] >= 0 && hi <= N, sb, 101);  // checks builds: key row inside K
                 if (kv[u]) {
                     const uint4* kr = reinterpret_cast<const uint4*>(K + ((size_t)jj[u] * H + h) * D);
 #pragma unroll
@@ -208,7 +208,10 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
         // a dropped group scores at most g_min + err(g_min) exactly (scaled); it matters if that reaches the
         // k-th best score found
         if (n_valid == LIST && g_min + ea + er * fabsf(g_min) >= kth * sc - fp32_err) {
-            if (lane == 0) redo_list[atomicAdd(&sb->n_redo, 1)] = (int)r;
+            if (lane == 0) {
+                const int pos = atomicAdd(&sb->n_redo, 1);
+                if (kmip_check(pos >= 0 && pos < n_rows, sb, 102)) redo_list[pos] = (int)r;  // checks builds: inside the list
+            }
         }
         warp_store_row(row, k, lane, topk_idx + (size_t)r * k, topk_score + (size_t)r * k);
     }

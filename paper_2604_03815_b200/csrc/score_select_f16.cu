@@ -496,7 +496,9 @@ score_select_f16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const int nloc = min(32, it.nrows - (qt * BM + quarter * 32));
                 for (int r = 0; r < nloc; ++r) {
                     const int srow = it.row0 + qt * BM + quarter * 32 + r;  // sweep order; the result goes to the row's own place
-                    const size_t o = ((size_t)(perm ? __ldg(perm + srow) : srow) * H + h) * LIST;
+                    const int orow = perm ? __ldg(perm + srow) : srow;
+                    if (!kmip_check(orow >= 0 && orow < n_total, sb, 103)) continue;  // checks builds: a row of the batch
+                    const size_t o = ((size_t)orow * H + h) * LIST;
                     for (int t = lane; t < LIST; t += 32) {
                         const uint32_t c = wl[t * 32 + r];
                         cand_word[o + t] = c ? wk[t * 32 + r] : 0xFFFFFFFFu;

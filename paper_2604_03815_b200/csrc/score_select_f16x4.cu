@@ -414,7 +414,9 @@ score_select_f16x4_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             uint32_t* wk_g = cand_word;
             if (!DUMP && rvalid) {
                 const int srow = it.row0 + local;
-                wk_g = cand_word + ((size_t)(perm ? __ldg(perm + srow) : srow) * H + h) * LIST;
+                const int orow = perm ? __ldg(perm + srow) : srow;
+                // checks builds: a row of the batch (a row that fails keeps writing to row 0's slots of the scratch list)
+                if (kmip_check(orow >= 0 && orow < n_total, sb, 103)) wk_g = cand_word + ((size_t)orow * H + h) * LIST;
             }
             __syncwarp();
             const int ntiles = (it.key_hi - it.key_lo + BN - 1) / BN;

@@ -278,3 +278,28 @@ def test_workspace_is_linear_in_n():
     # slot per (node, head), 6 bytes per node, work items
     rows = 1_000_000 * 4
     assert kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_FORWARD) < 2 * rows * 32 * 2 + rows * (24 * 6 + 4) + 8 * 1_000_000
+
+
+@pytest.mark.parametrize("d", [64, 32])
+def test_kth_score_near_zero_keeps_k_keys(d):
+    """Rows whose k-th best score is a tiny remainder of large cancelling terms: the tensor-core score and
+    the fp32 rescoring of the same key differ by far more than any margin RELATIVE to that score, and the
+    key that defines the k-th place must still come back (Algorithm 1 line 3 returns k keys whenever the
+    graph has k nodes): no padded slot, and the usual acceptance rule on every row."""
+    k, H, n = 8, 2, 600
+    w = wl.iid_workload("s", 6100 + d, [n, n], H, d, k, wl.MODE_BF16_TC)
+    rng = np.random.default_rng(61)
+    u = np.full(d, 0.125, dtype=np.float32)
+    alt = np.where(np.arange(d) % 2 == 0, 1.0, -1.0).astype(np.float32)
+    w.Q[:] = wl.round_to_bf16(u[None, None, :] + 0.01 * rng.standard_normal(w.Q.shape).astype(np.float32))
+    K = -u[None, None, :] * rng.uniform(0.5, 1.5, size=(w.N, H, 1)).astype(np.float32)          # clearly negative scores
+    for g0 in (0, n):
+        K[g0 + 3:g0 + 3 + (k - 1)] = 2.0 * u                                                      # k-1 clearly positive keys
+        near = g0 + 50 + 9 * np.arange(24)                                                         # 24 keys that score about zero
+        K[near] = 4.0 * (u * alt)[None, None, :] + 2.0 ** -13 * rng.standard_normal((24, H, d)).astype(np.float32)
+    w.K[:] = wl.round_to_bf16(K)
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    idx = fb.topk_idx.cpu().numpy()
+    assert np.all(idx >= 0), f"{int((idx < 0).sum())} padded slots although every graph has more than k nodes"
+    pu.check_forward(w, fb)
