@@ -179,6 +179,43 @@ int kmip_attn_topk_mass(const void *Q, const void *K,
                         void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The full layer of Eq. 2 (Algorithm 1 with its "Require" line and line 8), bf16 tensor-core mode:
+ *   Q^h = X W_Q^h,  K^h = X W_K^h,  V^h = X W_V^h,  O^h = kMIP-Attn(Q^h, K^h, V^h) inside each graph,
+ *   Y = sum_h O^h W_O^h,
+ * and its backward pass with the selection held constant (Sec. 3.1).  The four projections and every
+ * product of the backward pass run on the tensor cores in the library's own kernels; the attention core
+ * is kmip_attn_forward / kmip_attn_backward.  All tensors are bf16 device memory, 16-byte aligned:
+ *   x [N, d_model];  w_q, w_k, w_v [H*d_head, d_model] (row h*d_head + c holds column c of W^h);
+ *   w_o [d_model, H*d_head];  y, d_y, d_x [N, d_model];  dw_* in the shapes of the weights.
+ * d_model must be a multiple of 8, 1 <= d_head <= 128, k <= 128.  A head width other than 16, 32, 64, 128 (the
+ * paper's own study uses 10) is zero-padded to the next of those, d_pad, inside the call, which leaves
+ * every inner product unchanged; the softmax still divides by sqrt(d_head).
+ * Saved between the two calls, owned by the caller: q, k, v, o : bf16 [N, H, d_pad]; topk_idx int32 [N, H, k];
+ * topk_score float [N, H, k] - written by kmip_layer_forward, read by kmip_layer_backward.
+ * workspace: kmip_layer_workspace_bytes(..., pass) bytes of scratch; its first 256 bytes are the status
+ * block kmip_last_status reads (device-side problems of the attention core are forwarded to it).
+ * Errors, asynchrony and ownership as for kmip_attn_forward; other modes are KMIP_ERR_UNSUPPORTED.
+ */
+typedef struct {
+    const void *x, *w_q, *w_k, *w_v, *w_o;   /* inputs */
+    void *q, *k, *v, *o;                     /* saved projections and attention output, [N, H, d_pad] */
+    int32_t *topk_idx;                       /* saved selection */
+    float *topk_score;
+    void *y;                                 /* forward output; unused by the backward pass */
+    const void *d_y;                         /* backward input; unused by the forward pass */
+    void *d_x, *dw_q, *dw_k, *dw_v, *dw_o;   /* backward outputs (fully overwritten) */
+} kmip_layer_tensors_t;
+
+int kmip_layer_workspace_bytes(int64_t N, int32_t G, int32_t d_model, int32_t H, int32_t d_head, int32_t k,
+                               int pass, size_t *bytes);
+int kmip_layer_forward(const kmip_layer_tensors_t *t, const int32_t *graph_offsets, int32_t G, int64_t N,
+                       int32_t d_model, int32_t H, int32_t d_head, int32_t k,
+                       void *workspace, size_t workspace_bytes, void *stream);
+int kmip_layer_backward(const kmip_layer_tensors_t *t, const int32_t *graph_offsets, int32_t G, int64_t N,
+                        int32_t d_model, int32_t H, int32_t d_head, int32_t k,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Size in bytes of the scratch array that is built into the library for
  * kmip_attn_forward_static_scratch (8 MiB; each GPU that loads the library holds it until the
  * process exits).

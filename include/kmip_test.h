@@ -65,6 +65,15 @@ int kmip_test_f16_scores(const void *Q, const void *K, int64_t N, int32_t H, int
                          float *scores, float *stats, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The dense product behind the layer's projections (Eq. 2) on its own:
+ *   C[M, N] = A[M, K] B[N, K]^T,  A and B bf16 row-major device memory with lda = ldb = K (a multiple of 8),
+ * C bf16 (out_f32 = 0) or fp32 (out_f32 = 1) row-major with ldc = N, fp32 accumulation on the tensor cores.
+ * workspace: at least 256 bytes (status block).  Errors as for kmip_attn_forward.
+ */
+int kmip_test_gemm_tn(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K, int out_f32,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Where the tensor-core sweep of the last kmip_attn_forward call on `workspace` put each query row,
  * so that tests can sample rows by their place in the sweep (work-item borders, the split tail of
  * the schedule) and not only by their row number.  Synchronises `stream`, then writes to HOST memory

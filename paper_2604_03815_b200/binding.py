@@ -38,6 +38,12 @@ class TestOptions(ctypes.Structure):
                 ("fp32_path", ctypes.c_int32)]
 
 
+class LayerTensors(ctypes.Structure):
+    """kmip_layer_tensors_t of include/kmip.h (device pointers)."""
+    _fields_ = [(n, ctypes.c_void_p) for n in ("x", "w_q", "w_k", "w_v", "w_o", "q", "k", "v", "o", "topk_idx", "topk_score",
+                                                "y", "d_y", "d_x", "dw_q", "dw_k", "dw_v", "dw_o")]
+
+
 class KmipError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -81,6 +87,11 @@ def lib() -> ctypes.CDLL:
         L.kmip_profile_enable.argtypes = [ctypes.c_int]
         L.kmip_profile_read.restype = ctypes.c_int
         L.kmip_profile_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
+        L.kmip_layer_workspace_bytes.restype = ctypes.c_int
+        L.kmip_layer_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.c_int, ctypes.POINTER(sz)]
+        for fn in (L.kmip_layer_forward, L.kmip_layer_backward):
+            fn.restype = ctypes.c_int
+            fn.argtypes = [ctypes.POINTER(LayerTensors), P, i32, i64, i32, i32, i32, i32, P, sz, P]
         L.kmip_attn_sweep_counters.restype = ctypes.c_int
         L.kmip_attn_sweep_counters.argtypes = [P, P, ctypes.POINTER(ctypes.c_int64)]
         # kmip_test.h
@@ -88,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.kmip_test_tc_scores.argtypes = [P, P, i64, i32, i32, P, P, sz, P]
         L.kmip_test_f16_scores.restype = ctypes.c_int
         L.kmip_test_f16_scores.argtypes = [P, P, i64, i32, i32, P, P, P, sz, P]
+        L.kmip_test_gemm_tn.restype = ctypes.c_int
+        L.kmip_test_gemm_tn.argtypes = [P, P, P, i32, i32, i32, ctypes.c_int, P, sz, P]
         L.kmip_test_sweep_order.restype = ctypes.c_int
         L.kmip_test_sweep_order.argtypes = [P, i64, i32, i32, i32, i32, ctypes.c_int, P, ctypes.POINTER(i32), P]
         L.kmip_test_attn_forward.restype = ctypes.c_int
@@ -183,6 +196,31 @@ def kmip_attn_forward_static_scratch(Q, K, V, graph_offsets, k, mode, out, topk_
                                                       _ptr(device_status), _stream(stream)))
 
 
+def kmip_layer_workspace_bytes(N, G, d_model, H, d_head, k, pass_) -> int:
+    out = ctypes.c_size_t(0)
+    rc = lib().kmip_layer_workspace_bytes(N, G, d_model, H, d_head, k, pass_, ctypes.byref(out))
+    if rc != KMIP_OK:
+        raise KmipError(rc, "kmip_layer_workspace_bytes")
+    return int(out.value)
+
+
+def _layer_call(fn, tensors: dict, graph_offsets, N, d_model, H, d_head, k, workspace, stream):
+    t = LayerTensors(**{n: (None if v is None else v.data_ptr()) for n, v in tensors.items()})
+    G = 0 if graph_offsets is None else int(graph_offsets.numel()) - 1
+    return int(fn(ctypes.byref(t), _ptr(graph_offsets), G, N, d_model, H, d_head, k, _ptr(workspace),
+                  0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def kmip_layer_forward(tensors: dict, graph_offsets, N, d_model, H, d_head, k, workspace, stream=None) -> int:
+    """Eq. 2 forward: `tensors` maps the field names of kmip_layer_tensors_t to torch CUDA tensors (or None)."""
+    return _layer_call(lib().kmip_layer_forward, tensors, graph_offsets, N, d_model, H, d_head, k, workspace, stream)
+
+
+def kmip_layer_backward(tensors: dict, graph_offsets, N, d_model, H, d_head, k, workspace, stream=None) -> int:
+    """Eq. 2 backward with the saved selection; `tensors` as for kmip_layer_forward."""
+    return _layer_call(lib().kmip_layer_backward, tensors, graph_offsets, N, d_model, H, d_head, k, workspace, stream)
+
+
 def kmip_attn_backward(Q, K, V, graph_offsets, k, mode, out, d_out, topk_idx, topk_score, dQ, dK, dV,
                        workspace, stream=None) -> int:
     """Enqueue the backward pass; returns the library's status code (no exception, no sync)."""
@@ -236,6 +274,14 @@ def kmip_test_f16_scores(Q, K, scores, stats, workspace, stream=None) -> int:
     N, H, d = Q.shape
     return int(lib().kmip_test_f16_scores(_ptr(Q), _ptr(K), N, H, d, _ptr(scores), _ptr(stats), _ptr(workspace),
                                           workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def kmip_test_gemm_tn(A, B, C, workspace, stream=None) -> int:
+    """kmip_test.h: C[M, N] = A[M, K] B[N, K]^T (bf16 in, C bf16 or fp32) on the tensor cores."""
+    M, K = A.shape
+    N = B.shape[0]
+    return int(lib().kmip_test_gemm_tn(_ptr(A), _ptr(B), _ptr(C), M, N, K, 1 if C.dtype == torch.float32 else 0,
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def kmip_test_attn_forward(Q, K, V, graph_offsets, k, mode, out, topk_idx, topk_score, workspace, stream=None,

@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libkmip.so")
 LIB_CHECKS = os.path.join(HERE, "libkmip_checks.so")   # the same sources with -DKMIP_CHECKS (see include/kmip.h, kmip_build_flags)
-SOURCES = ["api.cu", "plan.cu", "reorder.cu", "prune.cu", "score_select_exact.cu", "score_select_fp32.cu", "score_select_tc.cu", "score_select_f16.cu", "score_select_f16x4.cu", "f16_convert.cu", "refine.cu", "refine_f16.cu", "epilogue.cu", "backward.cu", "topk_mass.cu",
+SOURCES = ["api.cu", "plan.cu", "reorder.cu", "prune.cu", "score_select_exact.cu", "score_select_fp32.cu", "score_select_tc.cu", "score_select_f16.cu", "score_select_f16x4.cu", "f16_convert.cu", "refine.cu", "refine_f16.cu", "epilogue.cu", "backward.cu", "topk_mass.cu", "gemm_tn.cu", "layer.cu",
            "static_scratch.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

@@ -225,6 +225,72 @@ int kmip_attn_topk_mass(const void* Q, const void* K, const int32_t* graph_offse
     return KMIP_OK;
 }
 
+static int check_layer(const kmip_layer_tensors_t* t, int64_t N, int32_t G, int32_t d_model, int32_t H, int32_t d_head, int32_t k,
+                       bool backward) {
+    if (d_head < 1 || d_head > 128 || d_model < 8 || (d_model & 7) || G < 0) return d_head > 128 ? KMIP_ERR_UNSUPPORTED : KMIP_ERR_INVALID_ARG;
+    const int rc = check_shape(N, H, layer_pad_width(d_head), k, KMIP_BF16_TC);
+    if (rc != KMIP_OK) return rc;
+    if (!t) return KMIP_ERR_INVALID_ARG;
+    const void* need_f[] = {t->x, t->w_q, t->w_k, t->w_v, t->w_o, t->q, t->k, t->v, t->o, t->topk_idx, t->topk_score};
+    for (const void* p : need_f)
+        if (!p || !aligned16(p)) return KMIP_ERR_INVALID_ARG;
+    if (!backward && (!t->y || !aligned16(t->y))) return KMIP_ERR_INVALID_ARG;
+    if (backward) {
+        const void* need_b[] = {t->d_y, t->d_x, t->dw_q, t->dw_k, t->dw_v, t->dw_o};
+        for (const void* p : need_b)
+            if (!p || !aligned16(p)) return KMIP_ERR_INVALID_ARG;
+    }
+    return KMIP_OK;
+}
+
+static LayerArgs layer_args(const kmip_layer_tensors_t* t, const int32_t* graph_offsets, int32_t G, int64_t N, int32_t d_model,
+                            int32_t H, int32_t d_head, int32_t k, void* workspace, void* stream) {
+    LayerArgs a{};
+    a.x = t->x; a.w_q = t->w_q; a.w_k = t->w_k; a.w_v = t->w_v; a.w_o = t->w_o;
+    a.q = t->q; a.k_proj = t->k; a.v = t->v; a.o = t->o;
+    a.topk_idx = t->topk_idx; a.topk_score = t->topk_score;
+    a.y = t->y; a.d_y = t->d_y;
+    a.d_x = t->d_x; a.dw_q = t->dw_q; a.dw_k = t->dw_k; a.dw_v = t->dw_v; a.dw_o = t->dw_o;
+    a.graph_offsets = graph_offsets; a.G = graph_offsets ? G : 1; a.N = N;
+    a.d_model = d_model; a.H = H; a.d_head = d_head; a.k = k;
+    a.ws = static_cast<unsigned char*>(workspace);
+    a.stream = static_cast<cudaStream_t>(stream);
+    return a;
+}
+
+int kmip_layer_workspace_bytes(int64_t N, int32_t G, int32_t d_model, int32_t H, int32_t d_head, int32_t k, int pass,
+                               size_t* bytes) {
+    if (!bytes || (pass != KMIP_PASS_FORWARD && pass != KMIP_PASS_BACKWARD)) return KMIP_ERR_INVALID_ARG;
+    if (d_head < 1 || d_model < 8 || (d_model & 7) || G < 0) return KMIP_ERR_INVALID_ARG;
+    if (d_head > 128) return KMIP_ERR_UNSUPPORTED;
+    const int rc = check_shape(N, H, layer_pad_width(d_head), k, KMIP_BF16_TC);
+    if (rc != KMIP_OK) return rc;
+    *bytes = plan_layer_workspace(N, G, d_model, H, d_head, k, pass).total;
+    return KMIP_OK;
+}
+
+int kmip_layer_forward(const kmip_layer_tensors_t* t, const int32_t* graph_offsets, int32_t G, int64_t N, int32_t d_model,
+                       int32_t H, int32_t d_head, int32_t k, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_layer(t, N, G, d_model, H, d_head, k, false);
+    if (rc != KMIP_OK) return rc;
+    if (N == 0) return KMIP_OK;
+    if ((graph_offsets != nullptr && G < 1) || !workspace || !aligned16(workspace)) return KMIP_ERR_INVALID_ARG;
+    if (workspace_bytes < plan_layer_workspace(N, graph_offsets ? G : 1, d_model, H, d_head, k, KMIP_PASS_FORWARD).total)
+        return KMIP_ERR_WORKSPACE;
+    return layer_forward(layer_args(t, graph_offsets, G, N, d_model, H, d_head, k, workspace, stream));
+}
+
+int kmip_layer_backward(const kmip_layer_tensors_t* t, const int32_t* graph_offsets, int32_t G, int64_t N, int32_t d_model,
+                        int32_t H, int32_t d_head, int32_t k, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_layer(t, N, G, d_model, H, d_head, k, true);
+    if (rc != KMIP_OK) return rc;
+    if (N == 0) return KMIP_OK;
+    if ((graph_offsets != nullptr && G < 1) || !workspace || !aligned16(workspace)) return KMIP_ERR_INVALID_ARG;
+    if (workspace_bytes < plan_layer_workspace(N, graph_offsets ? G : 1, d_model, H, d_head, k, KMIP_PASS_BACKWARD).total)
+        return KMIP_ERR_WORKSPACE;
+    return layer_backward(layer_args(t, graph_offsets, G, N, d_model, H, d_head, k, workspace, stream));
+}
+
 int kmip_last_status(const void* workspace, void* stream, int* device_status) {
     if (!workspace || !device_status) return KMIP_ERR_INVALID_ARG;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KMIP_ERR_CUDA;
@@ -288,6 +354,22 @@ int kmip_profile_read(double* stage_ms, int* calls) {
         }
     }
     g_prof.n_fwd = g_prof.n_bwd = 0;
+    return KMIP_OK;
+}
+
+int kmip_test_gemm_tn(const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int out_f32, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+    if (!A || !B || !C || !workspace || M < 1 || N < 1 || K < 8 || (K & 7)) return KMIP_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(C) || !aligned16(workspace)) return KMIP_ERR_INVALID_ARG;
+    if (workspace_bytes < kStatusBytes) return KMIP_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace, 0, kStatusBytes, st) != cudaSuccess) return KMIP_ERR_CUDA;
+    const void* As[3] = {A, A, A};
+    const void* Bs[3] = {B, B, B};
+    void* Cs[3] = {C, C, C};
+    if (launch_gemm_tn(As, K, Bs, K, Cs, nullptr, 1, 1, M, N, K, N, 0, 0, 0, 0, out_f32 != 0, static_cast<StatusBlock*>(workspace),
+                       st) != cudaSuccess)
+        return KMIP_ERR_CUDA;
     return KMIP_OK;
 }
 

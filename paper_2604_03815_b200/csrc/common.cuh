@@ -323,4 +323,38 @@ cudaError_t launch_softmax_gather(const FwdArgs& a);
 // ev (optional): three events recorded after the rows, inverse-index and segment stages
 cudaError_t launch_backward(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev);
 
+// gemm_tn.cu: C = scale * A B^T on the tensor cores (bf16 operands with K contiguous, fp32 accumulation); see there
+cudaError_t launch_gemm_tn(const void* const* A, int lda, const void* const* B, int ldb, void* const* C, const float* scale,
+                           int n_batch, int n_kseg, int M, int N, int K, int ldc, int row_pad, int row_real, int col_pad,
+                           int col_real, bool out_f32, StatusBlock* sb, cudaStream_t stream);
+
+// layer.cu: the full layer of Eq. 2 (bf16).  All pointers are device memory.
+struct LayerArgs {
+    const void *x, *w_q, *w_k, *w_v, *w_o;  // [N, d_model], [H*d_head, d_model] x 3, [d_model, H*d_head]
+    void *q, *k_proj, *v, *o;               // [N, H, d_pad]: written by the forward pass, read by the backward pass
+    int32_t* topk_idx;                      // [N, H, k]
+    float* topk_score;                      // [N, H, k]
+    void* y;                                // forward: [N, d_model]
+    const void* d_y;                        // backward: upstream gradient [N, d_model]
+    void *d_x, *dw_q, *dw_k, *dw_v, *dw_o;  // backward: gradients in the shapes of x and the weights
+    const int32_t* graph_offsets;
+    int32_t G;
+    int64_t N;
+    int32_t d_model, H, d_head, k;
+    unsigned char* ws;
+    cudaStream_t stream;
+};
+struct LayerWorkspace {
+    size_t wq_pad, wk_pad, wv_pad, wo_pad;         // padded weights
+    size_t wqT, wkT, wvT, woT;                     // their transposes (backward)
+    size_t d_o, d_q, d_k, d_v;                     // [N, H*d_pad] gradients around the attention core
+    size_t xT, dyT, oT, dqT, dkT, dvT;             // transposed activations for the weight gradients
+    size_t attn, attn_bytes;                       // workspace of the attention call
+    size_t total;
+};
+int layer_pad_width(int d_head);
+LayerWorkspace plan_layer_workspace(int64_t N, int32_t G, int32_t d_model, int32_t H, int32_t d_head, int32_t k, int pass);
+int layer_forward(const LayerArgs& a);   // kmip_status_t
+int layer_backward(const LayerArgs& a);
+
 }  // namespace kmip

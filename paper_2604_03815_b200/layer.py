@@ -2,11 +2,12 @@
 "Require" line and line 8): Q, K, V projections of the node features in front of the attention
 core and the output projection sum_h O^h W_O^h behind it, as a torch module with autograd.
 
-The attention core (scores, top-k, softmax, gather-V and its sparse backward) runs in the
-library's kernels through the two C-ABI calls; the four projections are plain dense GEMMs and
-use torch's (library GEMMs are what the paper's own implementation uses there too).  The
-selection is held constant in the backward pass (Sec. 3.1): gradients flow through the k kept
-scores only.
+In bfloat16 without attention dropout or pruning the whole layer - projections, attention core,
+output projection and every product of the backward pass - runs in the library's kernels through
+kmip_layer_forward / kmip_layer_backward (the projections on the tensor cores, csrc/gemm_tn.cu).
+Otherwise (float32, dropout, the pruned mode) the attention core runs through kmip_attn_forward /
+kmip_attn_backward and the four projections are torch's dense GEMMs.  The selection is held constant
+in the backward pass (Sec. 3.1): gradients flow through the k kept scores only.
 """
 import math
 
@@ -59,6 +60,56 @@ class KMIPAttentionFunction(torch.autograd.Function):
         return bb.dQ, bb.dK, bb.dV, None, None, None, None, None
 
 
+class KMIPLayerFunction(torch.autograd.Function):
+    """y = sum_h kMIP-Attn(x W_Q^h, x W_K^h, x W_V^h) W_O^h, bf16, through kmip_layer_forward / kmip_layer_backward."""
+
+    @staticmethod
+    def forward(ctx, x, w_q, w_k, w_v, w_o, graph_offsets, H, d_head, k):
+        x, w_q, w_k, w_v, w_o = (t.contiguous() for t in (x, w_q, w_k, w_v, w_o))
+        N, d_model = x.shape
+        d_pad = next(w for w in (16, 32, 64, 128) if w >= d_head)
+        G = 1 if graph_offsets is None else int(graph_offsets.numel()) - 1
+        dev = x.device
+        mk = lambda *shape, dtype=torch.bfloat16: torch.empty(shape, dtype=dtype, device=dev)
+        t = {"x": x, "w_q": w_q, "w_k": w_k, "w_v": w_v, "w_o": w_o,
+             "q": mk(N, H, d_pad), "k": mk(N, H, d_pad), "v": mk(N, H, d_pad), "o": mk(N, H, d_pad),
+             "topk_idx": mk(N, H, k, dtype=torch.int32), "topk_score": mk(N, H, k, dtype=torch.float32),
+             "y": mk(N, d_model), "d_y": None, "d_x": None, "dw_q": None, "dw_k": None, "dw_v": None, "dw_o": None}
+        ws = torch.empty(kb.kmip_layer_workspace_bytes(N, G, d_model, H, d_head, k, kb.PASS_FORWARD), dtype=torch.uint8, device=dev)
+        rc = kb.kmip_layer_forward(t, graph_offsets, N, d_model, H, d_head, k, ws)
+        if rc != kb.KMIP_OK:
+            raise kb.KmipError(rc, "kmip_layer_forward")
+        if N > 0:
+            st = kb.kmip_last_status(ws)     # the workspace is released right after, so device problems surface here
+            if st != kb.KMIP_OK:
+                raise kb.KmipError(st, "kmip_layer_forward (device)")
+        ctx.save_for_backward(x, w_q, w_k, w_v, w_o, t["q"], t["k"], t["v"], t["o"], t["topk_idx"], t["topk_score"])
+        ctx.meta = (graph_offsets, H, d_head, k)
+        ctx.mark_non_differentiable(t["topk_idx"])
+        return t["y"], t["topk_idx"]
+
+    @staticmethod
+    def backward(ctx, d_y, _d_idx):
+        x, w_q, w_k, w_v, w_o, q, kk, v, o, idx, score = ctx.saved_tensors
+        graph_offsets, H, d_head, k = ctx.meta
+        N, d_model = x.shape
+        G = 1 if graph_offsets is None else int(graph_offsets.numel()) - 1
+        t = {"x": x, "w_q": w_q, "w_k": w_k, "w_v": w_v, "w_o": w_o, "q": q, "k": kk, "v": v, "o": o,
+             "topk_idx": idx, "topk_score": score, "y": None, "d_y": d_y.contiguous().to(torch.bfloat16),
+             "d_x": torch.empty_like(x), "dw_q": torch.empty_like(w_q), "dw_k": torch.empty_like(w_k),
+             "dw_v": torch.empty_like(w_v), "dw_o": torch.empty_like(w_o)}
+        ws = torch.empty(kb.kmip_layer_workspace_bytes(N, G, d_model, H, d_head, k, kb.PASS_BACKWARD), dtype=torch.uint8,
+                         device=x.device)
+        rc = kb.kmip_layer_backward(t, graph_offsets, N, d_model, H, d_head, k, ws)
+        if rc != kb.KMIP_OK:
+            raise kb.KmipError(rc, "kmip_layer_backward")
+        if N > 0:
+            st = kb.kmip_last_status(ws)
+            if st != kb.KMIP_OK:
+                raise kb.KmipError(st, "kmip_layer_backward (device)")
+        return t["d_x"], t["dw_q"], t["dw_k"], t["dw_v"], t["dw_o"], None, None, None, None
+
+
 class KMIPSelfAttention(torch.nn.Module):
     """x [N, d_model] -> [N, d_model]: per head h, Q^h = x W_Q^h, K^h = x W_K^h, V^h = x W_V^h,
     O^h = kMIP-Attn(Q^h, K^h, V^h) restricted to each graph, y = sum_h O^h W_O^h (Eq. 2).
@@ -103,6 +154,13 @@ class KMIPSelfAttention(torch.nn.Module):
 
     def forward(self, x, graph_offsets=None, return_indices=False):
         N = x.shape[0]
+        drop_now = self.attn_dropout if self.training else 0.0
+        if (self.mode == kb.KMIP_BF16_TC and drop_now == 0.0 and self.w_q.bias is None and self.d_model % 8 == 0
+                and x.dtype == torch.bfloat16):
+            # the whole layer in the library's kernels
+            y, idx = KMIPLayerFunction.apply(x, self.w_q.weight, self.w_k.weight, self.w_v.weight, self.w_o.weight,
+                                             graph_offsets, self.H, self.d, self.k)
+            return (y, idx) if return_indices else y
         q = self.w_q(x).view(N, self.H, self.d)
         k = self.w_k(x).view(N, self.H, self.d)
         v = self.w_v(x).view(N, self.H, self.d)

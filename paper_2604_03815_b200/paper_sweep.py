@@ -4,8 +4,11 @@ inference pass (forward) and of a training pass (forward + backward) and peak de
 N = 10^(i/2).  The library stores head widths 16/32/64/128, so d_K = 10 is zero-padded to 16.
 
     python -m paper_2604_03815_b200.paper_sweep [--min-exp 8] [--max-exp 13] [--mode bf16|fp32] [--reps 3]
+                                                [--k 10] [--json out.json]
 
-Prints one JSON line per size and a markdown table at the end.  The paper's own figures (A100-40GB,
+--k changes the number of keys kept (the paper's appendix "Additional results", "Influence of k", reports
+whole-model epoch times for k up to 100, where its implementation slows down sharply).
+Prints one JSON line per size and a markdown table at the end; --json also writes the rows to a file.  The paper's own figures (A100-40GB,
 fp32 on CUDA cores, Tables of App. J.1 / K) are printed beside ours as context: another GPU,
 another precision, not a target.
 """
@@ -24,25 +27,25 @@ PAPER_SECONDS = {
 }
 
 
-def run_size(N, mode, reps):
+def run_size(N, mode, reps, k=10):
     import torch
 
     dev = torch.device("cuda", torch.cuda.current_device())
-    w = wl.padded_workload(f"paper_sweep_{N}", 7, N, 1, 10, 16, 10, mode)
+    w = wl.padded_workload(f"paper_sweep_{N}", 7, N, 1, 10, 16, k, mode)
     dt = kb.storage_dtype(mode)
     torch.cuda.empty_cache()
     torch.cuda.reset_peak_memory_stats(dev)
     Q, K, V, dO = (torch.from_numpy(getattr(w, n)).to(dev, dt) for n in ("Q", "K", "V", "dOut"))
     offs = torch.from_numpy(w.graph_offsets).to(dev)
-    fb = kb.ForwardBuffers(N, 1, 1, 16, 10, mode, dev)
-    bb = kb.BackwardBuffers(N, 1, 1, 16, 10, mode, dev)
+    fb = kb.ForwardBuffers(N, 1, 1, 16, k, mode, dev)
+    bb = kb.BackwardBuffers(N, 1, 1, 16, k, mode, dev)
 
     def fwd():
-        rc = kb.kmip_attn_forward(Q, K, V, offs, 10, mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace)
+        rc = kb.kmip_attn_forward(Q, K, V, offs, k, mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace)
         assert rc == kb.KMIP_OK, kb.status_string(rc)
 
     def bwd():
-        rc = kb.kmip_attn_backward(Q, K, V, offs, 10, mode, fb.out, dO, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK,
+        rc = kb.kmip_attn_backward(Q, K, V, offs, k, mode, fb.out, dO, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK,
                                    bb.dV, bb.workspace)
         assert rc == kb.KMIP_OK, kb.status_string(rc)
 
@@ -63,8 +66,8 @@ def run_size(N, mode, reps):
     t_inf = timed(fwd)
     t_train = timed(lambda: (fwd(), bwd()))
     peak = torch.cuda.max_memory_allocated(dev)
-    ref = PAPER_SECONDS.get(N, (None, None))
-    return {"N": N, "mode": "bf16" if mode == wl.MODE_BF16_TC else "fp32", "d_K": 10, "stored_d": 16, "k": 10,
+    ref = PAPER_SECONDS.get(N, (None, None)) if k == 10 else (None, None)
+    return {"N": N, "mode": "bf16" if mode == wl.MODE_BF16_TC else "fp32", "d_K": 10, "stored_d": 16, "k": k,
             "inference_s": t_inf, "training_s": t_train, "scores_per_s_inference": float(N) * N / t_inf,
             "peak_device_bytes": int(peak), "paper_a100_fp32_inference_s": ref[0], "paper_a100_fp32_training_s": ref[1]}
 
@@ -75,14 +78,19 @@ def main():
     ap.add_argument("--max-exp", type=int, default=13, help="largest N = 10^(max_exp/2); 14 = ten million nodes")
     ap.add_argument("--mode", choices=["bf16", "fp32"], default="bf16")
     ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--k", type=int, default=10, help="keys kept per query (the paper's sweep uses 10)")
+    ap.add_argument("--json", default=None, help="also write the rows to this file")
     args = ap.parse_args()
     mode = wl.MODE_BF16_TC if args.mode == "bf16" else wl.MODE_FP32_EXACT
     rows = []
     for i in range(args.min_exp, args.max_exp + 1):
         N = int(round(10 ** (i / 2)))
-        r = run_size(N, mode, args.reps if i < 13 else 1)
+        r = run_size(N, mode, args.reps if i < 13 else 1, args.k)
         rows.append(r)
         print(json.dumps(r), flush=True)
+    if args.json:
+        with open(args.json, "w") as f:
+            json.dump(rows, f, indent=1)
     print("\n| N | inference | training | peak device memory | paper (A100-40GB, fp32): inference / training |")
     print("|---|---|---|---|---|")
     for r in rows:

@@ -100,3 +100,39 @@ def test_forward_only_use_surfaces_device_errors():
     with torch.no_grad():
         y = layer(x, good)          # the context is still usable
     assert torch.isfinite(y.float()).all()
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (300, 200, 72), (1000, 384, 128), (130, 70, 8), (5, 515, 200),
+                                   (257, 129, 4104)])
+def test_projection_gemm_against_fp64(M, N, K):
+    """The tensor-core product behind the projections: ragged tile edges in all three dimensions, several
+    K blocks (the ring of shared-memory stages wraps), fp32 and bf16 outputs."""
+    from paper_2604_03815_b200 import binding as kb
+    g = torch.Generator(device="cpu").manual_seed(M * 7 + N * 3 + K)
+    A = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    B = torch.randn(N, K, generator=g).to(torch.bfloat16)
+    ref = A.double() @ B.double().T
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    for dt, tol in ((torch.float32, 1e-5), (torch.bfloat16, 2.0 ** -8)):
+        C = torch.full((M, N), float("nan"), dtype=dt, device="cuda")
+        assert kb.kmip_test_gemm_tn(A.cuda(), B.cuda(), C, ws) == kb.KMIP_OK
+        assert kb.kmip_last_status(ws) == kb.KMIP_OK
+        got = C.double().cpu()
+        assert torch.isfinite(got).all()
+        assert float((got - ref).abs().max()) <= tol * max(1.0, float(ref.abs().max())) + 1e-4 * np.sqrt(K) * (dt == torch.float32)
+
+
+def test_layer_calls_reject_bad_arguments():
+    from paper_2604_03815_b200 import binding as kb
+    with pytest.raises(kb.KmipError) as e:
+        kb.kmip_layer_workspace_bytes(1000, 1, 60, 2, 16, 8, kb.PASS_FORWARD)      # d_model not a multiple of 8
+    assert e.value.status == kb.KMIP_ERR_INVALID_ARG
+    with pytest.raises(kb.KmipError) as e:
+        kb.kmip_layer_workspace_bytes(1000, 1, 64, 2, 200, 8, kb.PASS_FORWARD)     # head wider than 128
+    assert e.value.status == kb.KMIP_ERR_UNSUPPORTED
+    f = kb.kmip_layer_workspace_bytes(100_000, 1, 128, 4, 32, 16, kb.PASS_FORWARD)
+    b = kb.kmip_layer_workspace_bytes(100_000, 1, 128, 4, 32, 16, kb.PASS_BACKWARD)
+    attn_f = kb.kmip_attn_workspace_bytes(100_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_FORWARD)
+    attn_b = kb.kmip_attn_workspace_bytes(100_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
+    assert attn_f < f < attn_f + (1 << 20)                                          # + four padded weight copies
+    assert attn_b + 10 * 100_000 * 128 * 2 <= b < attn_b + 10 * 100_008 * 128 * 2 + (1 << 21)   # + ten [N, 128] bf16 arrays
