@@ -31,7 +31,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 FWD_LAUNCHES = 5            # regroup keys, plan, score+select sweep, rescoring, softmax+gather-V
 F16_FWD_LAUNCHES = 8        # plan, norm maxima, K and Q conversions, prefilter sweep, rescoring, redo pass, softmax+gather-V
 REORDER_LAUNCHES = 3        # tensor-core mode from 32768 nodes on: locality codes, per-graph sort, permuted copy of Q
-BWD_LAUNCHES = 8            # rows, histogram, 3 scan kernels, fill, 2 segment kernels
+BWD_LAUNCHES = 9            # rows, partition (count, 3 scan kernels, scatter), bucket sort (writes the list offsets), 2 segment kernels
 
 
 def load_peaks():

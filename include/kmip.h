@@ -77,8 +77,9 @@ typedef enum {
  * needs for this problem size.  Linear in N*H*(k + d): the N x N score matrix of Algorithm 1
  * line 2 is never stored (Sec. 3.1, App. F).  Forward: one bf16 copy of K regrouped by head and, from
  * 32768 nodes on, one of Q in the sweep's row order plus 6 bytes per node
- * (tensor-core mode only) plus the work list; backward: 24 bytes per selected pair plus
- * 12 bytes per (node, head).  Host only, no CUDA call.
+ * (tensor-core mode only), for head widths up to 32 and k <= 32 also 6 bytes per kept candidate group
+ * (16, 24 or 48 per (node, head)), plus the work list; backward: 40 bytes per selected pair, 12 bytes per
+ * (node, head) and a 39 MB table.  Host only, no CUDA call.
  */
 int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k,
                               int mode, int pass, size_t *bytes);
@@ -117,8 +118,10 @@ int kmip_attn_forward(const void *Q, const void *K, const void *V,
  * Q, K; `out` is accepted for symmetry with autograd interfaces and may be NULL.
  * Outputs (fully overwritten): dQ, dK, dV.  graph_offsets and G are not needed by the
  * arithmetic (indices are global) and may be NULL / 0.
- * dK and dV are sums over an unordered list of hits: results are reproducible to fp32
- * rounding of the summation order, not bit for bit.
+ * dK and dV are sums over each key's list of hits in query order (the lists are built by a stable sort,
+ * without atomics), so the same inputs give the same gradients bit for bit on every run (up to 2^24
+ * (node, head) pairs; beyond that the lists are filled with atomic counters and the sums are
+ * reproducible to fp32 rounding only).
  */
 int kmip_attn_backward(const void *Q, const void *K, const void *V,
                        const int32_t *graph_offsets, int32_t G, int64_t N,

@@ -206,24 +206,275 @@ scan_write_kernel(int* __restrict__ counts, long long n, const int* __restrict__
     }
 }
 
-// A hit record of the key-major lists: everything the segment reduction needs about one selected
-// pair in one 16-byte load - the query row, its softmax weight p (times the dropout factor) and its
-// score gradient dS - instead of a pair id that would cost two more scattered 4-byte reads per hit.
-__global__ void fill_kernel(const int32_t* __restrict__ topk_idx, long long n_pairs, int N, int H, int k,
-                            const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
-                            const int* __restrict__ seg_off, int* __restrict__ cursor, int4* __restrict__ hits,
-                            StatusBlock* __restrict__ sb) {
+// In-place exclusive scan of n ints given the scanned sums of its 4096-item blocks (scan_block_sums_kernel,
+// scan_block_offsets_kernel).
+__global__ void __launch_bounds__(kScanThreads)
+scan_inplace_kernel(int* __restrict__ v, long long n, const int* __restrict__ block_sums) {
+    __shared__ int s_warp[32];
+    const long long base = (long long)blockIdx.x * kScanItemsPerBlock + (long long)threadIdx.x * kScanPerThread;
+    int c[kScanPerThread];
+    int t = 0;
+#pragma unroll
+    for (int u = 0; u < kScanPerThread; ++u) {
+        c[u] = (base + u < n) ? v[base + u] : 0;
+        t += c[u];
+    }
+    int total;
+    int off = block_sums[blockIdx.x] + block_exclusive_scan_1024(t, s_warp, total);
+#pragma unroll
+    for (int u = 0; u < kScanPerThread; ++u) {
+        if (base + u < n) v[base + u] = off;
+        off += c[u];
+    }
+}
+
+// ---- hit lists by a stable radix sort --------------------------------------------------------------
+// A hit record is everything the segment reduction needs about one selected pair in one 16-byte load:
+// {query row, softmax weight p (times the dropout factor), score gradient dS, (key, head) number}.  The
+// The records are sorted by (key, head) number in two stable steps, and the pairs start out in query
+// order, so each key's list ends up ordered by query row - the same order on every run, which makes the
+// sums of the segment stage reproducible bit for bit.  Pairs without a key (padding slots) get the number
+// n_rows and sort behind every list.
+//   partition  by the high digit of the number into buckets of 2^lo consecutive numbers: kRadixSlots warps
+//              own contiguous ranges of the pairs; each counts the digits of its range, an exclusive scan
+//              over (digit, slot) turns the counts into start offsets, and each warp walks its range again,
+//              32 records at a time, ranks equal digits by lane with a match vote and advances its own
+//              offsets - no atomics, so nothing depends on timing.  This is the one pass that scatters
+//              16-byte records over the whole buffer.
+//   buckets    one block per bucket sorts its records (a few hundred KB, served by L2) by the low digit
+//              with the same count / scan / ranked walk, its eight warps owning contiguous parts.
+struct RadixSrc {
+    const int32_t* topk_idx;  // first pass: the records are built from the pairs
+    const float* ws_p;
+    const float* ws_ds;
+    const int4* recs;         // later passes
+    int N, H, k;
+    int n_rows;
+};
+
+template <bool FIRST>
+__device__ __forceinline__ int4 radix_load(const RadixSrc& s, long long e) {
+    if (!FIRST) return __ldg(s.recs + e);
+    const int j = __ldg(s.topk_idx + e);
+    const long long r = e / s.k;  // query * H + head
+    const int key = (j >= 0 && j < s.N) ? j * s.H + (int)(r % s.H) : s.n_rows;
+    return make_int4((int)(r / s.H), __float_as_int(__ldg(s.ws_p + e)), __float_as_int(__ldg(s.ws_ds + e)), key);
+}
+
+// Per-warp digit counters are 16 bits wide (a warp's range holds fewer than 65536 records), two to a word.
+template <bool FIRST>
+__global__ void __launch_bounds__(kRadixWarps * 32)
+radix_count_kernel(const RadixSrc src, long long n, long long per_slot, int shift, int bins, int* __restrict__ table) {
+    extern __shared__ unsigned s_hist[];  // [kRadixWarps][bins / 2]
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int words = bins / 2;
+    for (int x = threadIdx.x; x < kRadixWarps * words; x += blockDim.x) s_hist[x] = 0u;
+    __syncthreads();
+    const int slot = blockIdx.x * kRadixWarps + w;
+    const long long lo = (long long)slot * per_slot, hi = min(n, lo + per_slot);
+    unsigned* hist = s_hist + w * words;
+    constexpr int U = 8;  // loads in flight per lane
+    for (long long e0 = lo; e0 < hi; e0 += 32 * U) {
+        int key[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long e = e0 + u * 32 + lane;
+            key[u] = -1;
+            if (e < hi) {
+                if (FIRST) {
+                    const int j = __ldg(src.topk_idx + e);
+                    key[u] = (j >= 0 && j < src.N) ? j * src.H + (int)((e / src.k) % src.H) : src.n_rows;
+                } else {
+                    key[u] = __ldg(reinterpret_cast<const int*>(src.recs + e) + 3);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (key[u] >= 0) {
+                const int d = (key[u] >> shift) & (bins - 1);
+                atomicAdd(hist + (d >> 1), 1u << (16 * (d & 1)));  // shared memory; the counts do not depend on the order
+            }
+        }
+    }
+    __syncthreads();
+    for (int x = threadIdx.x; x < kRadixWarps * bins; x += blockDim.x) {
+        const int ww = x / bins, d = x % bins;
+        table[(size_t)d * kRadixSlots + blockIdx.x * kRadixWarps + ww] = (int)((s_hist[ww * words + (d >> 1)] >> (16 * (d & 1))) & 0xFFFFu);
+    }
+}
+
+template <bool FIRST>
+__global__ void __launch_bounds__(kRadixWarps * 32)
+radix_scatter_kernel(const RadixSrc src, long long n, long long per_slot, int shift, int bins, const int* __restrict__ table,
+                     int4* __restrict__ dst, StatusBlock* __restrict__ sb) {
+    extern __shared__ unsigned s_hist[];  // viewed as unsigned short [kRadixWarps][bins]: records of each digit placed so far
+    unsigned short* s_cnt = reinterpret_cast<unsigned short*>(s_hist);
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int x = threadIdx.x; x < kRadixWarps * bins / 2; x += blockDim.x) s_hist[x] = 0u;
+    __syncthreads();
+    const int slot = blockIdx.x * kRadixWarps + w;
+    const long long lo = (long long)slot * per_slot, hi = min(n, lo + per_slot);
+    unsigned short* cnt = s_cnt + w * bins;
+    const int* start = table + slot;  // start[d * kRadixSlots]: where this warp's records of digit d begin
+    const unsigned lt = (1u << lane) - 1u;
+    constexpr int U = 8;  // records loaded ahead per lane; they are placed in order, 32 at a time
+    for (long long e0 = lo; e0 < hi; e0 += 32 * U) {
+        int4 recs[U];
+        int base[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long e = e0 + u * 32 + lane;
+            recs[u] = make_int4(0, 0, 0, -1);
+            if (e < hi) recs[u] = radix_load<FIRST>(src, e);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            base[u] = recs[u].w >= 0 ? __ldg(start + (size_t)((recs[u].w >> shift) & (bins - 1)) * kRadixSlots) : 0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (e0 + u * 32 >= hi) break;  // warp-uniform
+            const int4 rec = recs[u];
+            const bool live = e0 + u * 32 + lane < hi;
+            // lanes past the end of the range vote with digits of their own, which match nobody
+            const int digit = live ? ((rec.w >> shift) & (bins - 1)) : bins + lane;
+            const unsigned same = __match_any_sync(0xFFFFFFFFu, digit);
+            if (live) {
+                const int placed = cnt[digit];
+                const long long pos = (long long)base[u] + placed + __popc(same & lt);
+                if (kmip_check(pos >= 0 && pos < n, sb, 104)) dst[pos] = rec;  // checks builds: inside the buffer
+                __syncwarp(same);
+                if ((same & lt) == 0u) cnt[digit] = (unsigned short)(placed + __popc(same));  // the group's first lane moves the digit on
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// Fallback beyond 2^24 (node, head) pairs, where the two-digit sort above would need tables of more than
+// 4096 digits: every pair takes the next free place of its list with an atomic counter.  The lists then hold
+// the same records in an order that depends on timing, so dK and dV are reproducible to fp32 rounding only.
+__global__ void fill_unordered_kernel(const int32_t* __restrict__ topk_idx, long long n_pairs, int N, int H, int k,
+                                      const float* __restrict__ ws_p, const float* __restrict__ ws_ds,
+                                      const int* __restrict__ seg_off, int* __restrict__ cursor, int4* __restrict__ hits,
+                                      StatusBlock* __restrict__ sb) {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_pairs) return;
     const int j = __ldg(topk_idx + e);
     if (j < 0 || j >= N) return;
     const long long r = e / k;  // query * H + head
-    const int h = (int)(r % H);
-    const size_t key = (size_t)j * H + h;
+    const size_t key = (size_t)j * H + (int)(r % H);
     const long long pos = (long long)seg_off[key] + atomicAdd(cursor + key, 1);
     if (!kmip_check(pos >= 0 && pos < n_pairs, sb, 104)) return;  // checks builds: inside the hit lists
-    hits[pos] =
-        make_int4((int)(r / H), __float_as_int(__ldg(ws_p + e)), __float_as_int(__ldg(ws_ds + e)), 0);
+    hits[pos] = make_int4((int)(r / H), __float_as_int(__ldg(ws_p + e)), __float_as_int(__ldg(ws_ds + e)), (int)key);
+}
+
+// Second step: the records of one bucket (high digit = blockIdx.x), src -> dst, ordered by the low digit and,
+// within a digit, in the order they have in src.  bucket_start[d * kRadixSlots] is where bucket d begins.  The low
+// digit of a number inside its bucket IS the (key, head) pair, so this kernel also knows where every list starts:
+// it writes seg_off (rows + 1 entries) and the list of long segments.
+constexpr int kBucketWarps = 8;
+__global__ void __launch_bounds__(kBucketWarps * 32)
+radix_bucket_kernel(const int4* __restrict__ src, int4* __restrict__ dst, const int* __restrict__ bucket_start, int n_buckets,
+                    long long n, int lo_bits, long long n_rows, int* __restrict__ seg_off, int* __restrict__ long_list,
+                    StatusBlock* __restrict__ sb) {
+    extern __shared__ int s_cnt[];  // [kBucketWarps][bins]: counts, then next free positions
+    __shared__ int s_tot[32];
+    __shared__ int s_carry;
+    const int bins = 1 << lo_bits;
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int d_hi = blockIdx.x;
+    const long long begin = bucket_start[(size_t)d_hi * kRadixSlots];
+    const long long end = d_hi + 1 < n_buckets ? (long long)bucket_start[(size_t)(d_hi + 1) * kRadixSlots] : n;
+    const long long len = end - begin;
+    for (int x = threadIdx.x; x < kBucketWarps * bins; x += blockDim.x) s_cnt[x] = 0;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    const long long per = ((len + kBucketWarps - 1) / kBucketWarps + 31) / 32 * 32;
+    const long long lo = begin + (long long)w * per, hi = min(end, lo + per);
+    int* cnt = s_cnt + w * bins;
+    constexpr int U = 8;
+    for (long long e0 = lo; e0 < hi; e0 += 32 * U) {
+        int key[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long e = e0 + u * 32 + lane;
+            key[u] = e < hi ? __ldg(reinterpret_cast<const int*>(src + e) + 3) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (key[u] >= 0) atomicAdd(cnt + (key[u] & (bins - 1)), 1);  // shared memory; counts do not depend on the order
+    }
+    __syncthreads();
+    // exclusive scan over (digit, warp): thread per digit across the warps, then the digit totals across the block
+    for (int d0 = 0; d0 < bins; d0 += blockDim.x) {
+        const int d = d0 + threadIdx.x;
+        int tot = 0;
+        if (d < bins) {
+#pragma unroll
+            for (int ww = 0; ww < kBucketWarps; ++ww) {
+                const int c = s_cnt[ww * bins + d];
+                s_cnt[ww * bins + d] = tot;  // warp ww's first record of this digit, relative to the digit's start
+                tot += c;
+            }
+        }
+        int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_tot[w] = incl;
+        __syncthreads();
+        if (w == 0) {
+            int v = lane < kBucketWarps ? s_tot[lane] : 0;
+#pragma unroll
+            for (int o = 1; o < kBucketWarps; o <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, v, o);
+                if (lane >= o) v += t;
+            }
+            if (lane < kBucketWarps) s_tot[lane] = v;  // inclusive over warps
+        }
+        __syncthreads();
+        const int digit_start = s_carry + (w ? s_tot[w - 1] : 0) + incl - tot;
+        if (d < bins) {
+#pragma unroll
+            for (int ww = 0; ww < kBucketWarps; ++ww) s_cnt[ww * bins + d] += digit_start;
+            // this digit is (key, head) pair number d_hi * bins + d: its list starts here and holds `tot` hits
+            const long long pair = (long long)d_hi * bins + d;
+            if (pair <= n_rows) seg_off[pair] = (int)(begin + digit_start);
+            if (pair < n_rows && tot > kLongSeg) long_list[atomicAdd(&sb->n_long, 1)] = (int)pair;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_carry += s_tot[kBucketWarps - 1];
+        __syncthreads();
+    }
+    // ranked walk, as in radix_scatter_kernel
+    const unsigned lt = (1u << lane) - 1u;
+    for (long long e0 = lo; e0 < hi; e0 += 32 * U) {
+        int4 recs[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long e = e0 + u * 32 + lane;
+            recs[u] = e < hi ? __ldg(src + e) : make_int4(0, 0, 0, -1);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (e0 + u * 32 >= hi) break;  // warp-uniform
+            const int4 rec = recs[u];
+            const bool live = e0 + u * 32 + lane < hi;
+            const int digit = live ? (rec.w & (bins - 1)) : bins + lane;
+            const unsigned same = __match_any_sync(0xFFFFFFFFu, digit);
+            if (live) {
+                const int base = cnt[digit];
+                const long long pos = begin + base + __popc(same & lt);
+                if (kmip_check(pos >= begin && pos < end, sb, 106)) dst[pos] = rec;  // checks builds: inside the bucket
+                __syncwarp(same);
+                if ((same & lt) == 0u) cnt[digit] = base + __popc(same);
+            }
+            __syncwarp();
+        }
+    }
 }
 
 // -------------------------------------------------------------------------------------- segments
@@ -380,14 +631,15 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     int* seg_off = reinterpret_cast<int*>(a.ws + w.seg_off);
     int* cursor = reinterpret_cast<int*>(a.ws + w.cursor_off);
     int4* hits = reinterpret_cast<int4*>(a.ws + w.pairs_off);
+    int4* tmp = reinterpret_cast<int4*>(a.ws + w.tmp_off);
+    int* table = reinterpret_cast<int*>(a.ws + w.table_off);
+    int* tblsum = reinterpret_cast<int*>(a.ws + w.tblsum_off);
     int* block_sums = reinterpret_cast<int*>(a.ws + w.blocksum_off);
     int* long_list = reinterpret_cast<int*>(a.ws + w.long_off);
     const T *Q = static_cast<const T*>(a.Q), *K = static_cast<const T*>(a.K), *V = static_cast<const T*>(a.V);
     const T* dOut = static_cast<const T*>(a.d_out);
     const float scale = 1.0f / sqrtf((float)a.d);
     cudaError_t err;
-
-    if ((err = cudaMemsetAsync(cursor, 0, sizeof(int) * (size_t)(n_rows + 1), a.stream)) != cudaSuccess) return err;
 
     const int row_blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 32);
     bwd_rows_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(
@@ -396,12 +648,40 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     if (ev) cudaEventRecord(ev[0], a.stream);
 
     const int pair_blocks = (int)((n_pairs + 255) / 256);
-    hist_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, cursor, sb);
-    scan_block_sums_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums);
-    scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(block_sums, w.scan_blocks);
-    scan_write_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums, seg_off, long_list, sb);
-    fill_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, ws_p, ws_ds, seg_off, cursor,
-                                                  hits, sb);
+    // the hit lists: stable partition of the pairs by the high digit of their (key, head) number, then a stable
+    // sort of every bucket by the low digit, which also writes the list offsets
+    {
+        int bits, lo_bits, hi_bits;
+        radix_digits(n_rows, bits, lo_bits, hi_bits);
+        const long long per_slot = ((n_pairs + kRadixSlots - 1) / kRadixSlots + 31) / 32 * 32;
+        if (bits > 2 * kRadixMaxBits || per_slot > 65535) {
+            // more than 16.7 million (node, head) pairs or 465 million selected pairs: unordered lists
+            if ((err = cudaMemsetAsync(cursor, 0, sizeof(int) * (size_t)(n_rows + 1), a.stream)) != cudaSuccess) return err;
+            hist_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, cursor, sb);
+            scan_block_sums_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums);
+            scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(block_sums, w.scan_blocks);
+            scan_write_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums, seg_off, long_list, sb);
+            fill_unordered_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, ws_p, ws_ds, seg_off,
+                                                                    cursor, hits, sb);
+        } else {
+            const int bins_hi = 1 << hi_bits, bins_lo = 1 << lo_bits;
+            const long long n_tab = (long long)bins_hi * kRadixSlots;
+            const int tab_blocks = (int)((n_tab + kScanItemsPerBlock - 1) / kScanItemsPerBlock);
+            const size_t smem_hi = (size_t)kRadixWarps * bins_hi * 2, smem_lo = (size_t)kBucketWarps * bins_lo * sizeof(int);
+            if ((err = cudaFuncSetAttribute(radix_count_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hi)) != cudaSuccess ||
+                (err = cudaFuncSetAttribute(radix_scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hi)) != cudaSuccess ||
+                (err = cudaFuncSetAttribute(radix_bucket_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lo)) != cudaSuccess)
+                return err;
+            RadixSrc src{a.topk_idx, ws_p, ws_ds, nullptr, (int)a.N, a.H, a.k, (int)n_rows};
+            radix_count_kernel<true><<<kRadixBlocks, kRadixWarps * 32, smem_hi, a.stream>>>(src, n_pairs, per_slot, lo_bits, bins_hi, table);
+            scan_block_sums_kernel<<<tab_blocks, kScanThreads, 0, a.stream>>>(table, n_tab, tblsum);
+            scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(tblsum, tab_blocks);
+            scan_inplace_kernel<<<tab_blocks, kScanThreads, 0, a.stream>>>(table, n_tab, tblsum);
+            radix_scatter_kernel<true><<<kRadixBlocks, kRadixWarps * 32, smem_hi, a.stream>>>(src, n_pairs, per_slot, lo_bits, bins_hi, table, tmp, sb);
+            radix_bucket_kernel<<<bins_hi, kBucketWarps * 32, smem_lo, a.stream>>>(tmp, hits, table, bins_hi, n_pairs, lo_bits, n_rows,
+                                                                                seg_off, long_list, sb);
+        }
+    }
     if (ev) cudaEventRecord(ev[1], a.stream);
 
     bwd_segments_kernel<T, D><<<row_blocks, kWarpsPerBlock * 32, 0, a.stream>>>(

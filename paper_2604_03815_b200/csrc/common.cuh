@@ -152,7 +152,10 @@ struct BwdWorkspace {
     size_t ds_off;        // float [N*H*k]   score gradients
     size_t seg_off;       // int   [N*H+1]   start of each (key, head) hit list
     size_t cursor_off;    // int   [N*H]     hit counts, then fill cursors
-    size_t pairs_off;     // int4  [N*H*k]   hit lists: records {query row, p, dS, 0}
+    size_t pairs_off;     // int4  [N*H*k]   hit lists: records {query row, p, dS, (key, head) number}
+    size_t tmp_off;       // int4  [N*H*k]   the other buffer of the radix passes that build them
+    size_t table_off;     // int   [high digits * kRadixSlots]  digit counts per (digit, slot), then offsets
+    size_t tblsum_off;    // int   block sums of the scan over that table
     size_t blocksum_off;  // int   [scan blocks]
     size_t long_off;      // int   [N*H]     ids of long segments
     size_t total;
@@ -161,6 +164,18 @@ struct BwdWorkspace {
 };
 
 constexpr int kScanItemsPerBlock = 4096;
+// The hit lists are built by a stable radix sort of the selected pairs by (key, head) number, so every list
+// comes out ordered by query row whatever the timing: kRadixSlots warps each own a contiguous range of pairs.
+constexpr int kRadixBlocks = 444, kRadixWarps = 16, kRadixSlots = kRadixBlocks * kRadixWarps;
+constexpr int kRadixMaxBits = 12, kRadixMaxBins = 1 << kRadixMaxBits;
+// digits of the two steps for `rows` (node, head) pairs: the numbers 0 .. rows (rows = "no key") split into a
+// high and a low digit; more than 2 * kRadixMaxBits bits are not sorted (unordered fallback)
+inline void radix_digits(long long rows, int& bits, int& lo_bits, int& hi_bits) {
+    bits = 1;
+    while ((1ll << bits) <= rows) ++bits;
+    lo_bits = bits / 2;
+    hi_bits = bits - lo_bits;
+}
 
 inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
     BwdWorkspace w;
@@ -177,6 +192,12 @@ inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
     w.seg_off = o;      o = region(o + 4 * (rows + 1));
     w.cursor_off = o;   o = region(o + 4 * (rows + 1));
     w.pairs_off = o;    o = region(o + 16 * pairs);
+    w.tmp_off = o;      o = region(o + 16 * pairs);
+    int bits, lo_bits, hi_bits;
+    radix_digits((long long)rows, bits, lo_bits, hi_bits);
+    const size_t bins_hi = bits <= 2 * kRadixMaxBits ? ((size_t)1 << hi_bits) : 1;
+    w.table_off = o;    o = region(o + 4 * bins_hi * kRadixSlots);
+    w.tblsum_off = o;   o = region(o + 4 * (bins_hi * kRadixSlots / kScanItemsPerBlock + 2));
     w.blocksum_off = o; o = region(o + 4 * (size_t)(w.scan_blocks + 1));
     w.long_off = o;     o = region(o + 4 * rows);
     w.total = o;

@@ -68,7 +68,9 @@ def test_workspace_bytes_host_only(kb):
     assert srows * 64 < sp < srows * 64 + (1 << 20)
     assert kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_BACKWARD) == b
     pairs = 500_000 * 4 * 32
-    assert 24 * pairs < b < 26 * pairs          # p, dS, 16-byte hit records: 24 bytes per selected pair + O(N*H)
+    # p, dS and two buffers of 16-byte hit records (the radix sort that orders them): 40 bytes per selected pair,
+    # 12 per (node, head), and a 39 MB table of digit counts
+    assert 40 * pairs < b < 40 * pairs + 14 * 500_000 * 4 + (40 << 20)
     for bad in [dict(d=24), dict(k=129), dict(mode=7)]:
         args = dict(N=1000, G=1, H=2, d=32, k=8, mode=kb.KMIP_BF16_TC)
         args.update(bad)

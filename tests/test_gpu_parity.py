@@ -273,7 +273,7 @@ def test_workspace_too_small_is_refused():
 def test_workspace_is_linear_in_n():
     a = kb.kmip_attn_workspace_bytes(100_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
     b = kb.kmip_attn_workspace_bytes(1_000_000, 1, 4, 32, 16, kb.KMIP_BF16_TC, kb.PASS_BACKWARD)
-    assert b < 10.5 * a and b < 1_000_000 * 4 * (6 * 16 + 4) * 4 + (1 << 20)   # 24 bytes per selected pair + per-row arrays
+    assert b < 10.5 * a and b < 1_000_000 * 4 * (10 * 16 + 4) * 4 + (160 << 20)   # 40 bytes per selected pair + per-row arrays + digit table (at most 4096 digits x 7104 warps x 4 bytes)
     # forward: 2-byte copies of K (regrouped) and Q (sweep order), the prefilter's 24 groups of 6 bytes and a redo
     # slot per (node, head), 6 bytes per node, work items
     rows = 1_000_000 * 4

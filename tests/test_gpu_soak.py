@@ -64,23 +64,72 @@ def test_random_shapes(seed, force_wide, cases):
 def test_large_runs_are_bit_identical(cfg, kw, pruned):
     """The selection is exact whatever the timing of the pipeline, so repeated runs on the same
     inputs must agree bit for bit; a run that read an accumulator or a key stage at the wrong
-    moment would not."""
+    moment would not.  The backward pass too: its hit lists are ordered by a stable sort, so dQ, dK and
+    dV of repeated runs are bit-identical as well."""
     w = wl.make_config(cfg, **kw)
     mode = kb.KMIP_BF16_TC_PRUNED if pruned else w.mode  # the pruned mode's key and row orders come from stable sorts
     dt = kb.storage_dtype(mode)
     Q, K, V = (torch.from_numpy(getattr(w, n)).to("cuda", dt) for n in "QKV")
     offs = torch.from_numpy(w.graph_offsets).cuda()
     fb = kb.ForwardBuffers(w.N, len(w.graph_offsets) - 1, w.H, w.d, w.k, mode)
+    bb = kb.BackwardBuffers(w.N, len(w.graph_offsets) - 1, w.H, w.d, w.k, mode)
+    dO = torch.from_numpy(w.dOut).to("cuda", dt)
     ref = None
     for _ in range(6):
         assert kb.kmip_attn_forward(Q, K, V, offs, w.k, mode, fb.out, fb.topk_idx, fb.topk_score, fb.workspace) == kb.KMIP_OK
+        assert kb.kmip_attn_backward(Q, K, V, offs, w.k, mode, fb.out, dO, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK, bb.dV,
+                                     bb.workspace) == kb.KMIP_OK
         torch.cuda.synchronize()
-        assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK
-        cur = (fb.topk_idx.clone(), fb.topk_score.clone(), fb.out.clone())
+        assert kb.kmip_last_status(fb.workspace) == kb.KMIP_OK and kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
+        cur = (fb.topk_idx.clone(), fb.topk_score.clone(), fb.out.clone(), bb.dQ.clone(), bb.dK.clone(), bb.dV.clone())
         if ref is None:
             ref = cur
         else:
             assert all(torch.equal(a, b) for a, b in zip(ref, cur))
+
+
+def test_backward_of_the_full_size_configs_is_bit_identical():
+    """Configs 4 and 5 at full size (64 and 102 million selected pairs; config 5's hub keys collect thousands
+    of hits each): three backward passes on the same saved selection give the same bits."""
+    for cfg in (4, 5):
+        w = wl.make_config(cfg)
+        dt = kb.storage_dtype(w.mode)
+        Q, K, V, dO = (torch.from_numpy(getattr(w, n)).to("cuda", dt) for n in ("Q", "K", "V", "dOut"))
+        offs = torch.from_numpy(w.graph_offsets).cuda()
+        fb = kb.forward(Q, K, V, offs, w.k, w.mode)
+        bb = kb.BackwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode)
+        ref = None
+        for _ in range(3):
+            assert kb.kmip_attn_backward(Q, K, V, offs, w.k, w.mode, fb.out, dO, fb.topk_idx, fb.topk_score, bb.dQ, bb.dK,
+                                         bb.dV, bb.workspace) == kb.KMIP_OK
+            assert kb.kmip_last_status(bb.workspace) == kb.KMIP_OK
+            cur = (bb.dQ.clone(), bb.dK.clone(), bb.dV.clone())
+            if ref is not None:
+                assert all(torch.equal(a, b) for a, b in zip(ref, cur))
+            ref = cur
+        del fb, bb
+
+
+def test_one_key_selected_by_every_query():
+    """The longest possible hit list: one key that every query of a 200 000-node graph selects (its key row
+    is a hundred times heavier than the rest).  The backward pass must stay correct - checked against the
+    oracle - and finish in a bounded time (one block reduces the list; measured about 10 ms)."""
+    from tests import parity_util as pu
+    w = wl.iid_workload("s", 9100, [200_000], 1, 32, 4, wl.MODE_BF16_TC)
+    w.Q[:] = np.abs(w.Q)
+    w.K[777] = np.float32(100.0) * np.abs(w.K[777])
+    w.K[:] = wl.round_to_bf16(w.K)
+    dev = pu.to_device(w)
+    fb = pu.run_forward(w, dev)
+    assert bool((fb.topk_idx[:, 0, 0] == 777).all())
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    bb = pu.run_backward(w, fb, dev)
+    e0.record()
+    bb = pu.run_backward(w, fb, dev)
+    e1.record()
+    torch.cuda.synchronize()
+    pu.check_backward(w, fb, bb)
+    assert e0.elapsed_time(e1) < 100.0, f"backward with a 200 000-hit list took {e0.elapsed_time(e1):.1f} ms"
 
 
 def test_random_small_shapes_against_the_oracle():
