@@ -264,7 +264,8 @@ __device__ __forceinline__ int4 radix_load(const RadixSrc& s, long long e) {
 // Per-warp digit counters are 16 bits wide (a warp's range holds fewer than 65536 records), two to a word.
 template <bool FIRST>
 __global__ void __launch_bounds__(kRadixWarps * 32)
-radix_count_kernel(const RadixSrc src, long long n, long long per_slot, int shift, int bins, int* __restrict__ table) {
+radix_count_kernel(const RadixSrc src, long long n, long long per_slot, int shift, int bins, int* __restrict__ table,
+                   StatusBlock* __restrict__ sb) {
     extern __shared__ unsigned s_hist[];  // [kRadixWarps][bins / 2]
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int words = bins / 2;
@@ -283,6 +284,7 @@ radix_count_kernel(const RadixSrc src, long long n, long long per_slot, int shif
             if (e < hi) {
                 if (FIRST) {
                     const int j = __ldg(src.topk_idx + e);
+                    kmip_check(j < src.N, sb, 105);  // checks builds: an index the forward pass cannot have written (ignored either way)
                     key[u] = (j >= 0 && j < src.N) ? j * src.H + (int)((e / src.k) % src.H) : src.n_rows;
                 } else {
                     key[u] = __ldg(reinterpret_cast<const int*>(src.recs + e) + 3);
@@ -673,7 +675,7 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
                 (err = cudaFuncSetAttribute(radix_bucket_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lo)) != cudaSuccess)
                 return err;
             RadixSrc src{a.topk_idx, ws_p, ws_ds, nullptr, (int)a.N, a.H, a.k, (int)n_rows};
-            radix_count_kernel<true><<<kRadixBlocks, kRadixWarps * 32, smem_hi, a.stream>>>(src, n_pairs, per_slot, lo_bits, bins_hi, table);
+            radix_count_kernel<true><<<kRadixBlocks, kRadixWarps * 32, smem_hi, a.stream>>>(src, n_pairs, per_slot, lo_bits, bins_hi, table, sb);
             scan_block_sums_kernel<<<tab_blocks, kScanThreads, 0, a.stream>>>(table, n_tab, tblsum);
             scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(tblsum, tab_blocks);
             scan_inplace_kernel<<<tab_blocks, kScanThreads, 0, a.stream>>>(table, n_tab, tblsum);

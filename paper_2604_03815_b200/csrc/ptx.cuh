@@ -314,5 +314,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// 16-byte asynchronous copy global -> shared that bypasses L1 (both addresses 16-byte aligned); copies issued by a
+// thread complete in groups: commit closes a group, wait<N> returns when all but the newest N groups have landed
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 }  // namespace ptx
 }  // namespace kmip

@@ -2,7 +2,7 @@
 //
 // score_select_f16.cu leaves, for every (query, head), the L best 8-key groups by the fp16 maximum
 // of their tensor-core scores (L = k + slack).  This kernel turns them into the exact answer:
-//   1. m_k = k-th largest group maximum.  The k groups at or above it each hold a key whose exact score
+//   1. m_k = k-th largest group maximum (a 16-step search over the bits of the half-precision value).  The k groups at or above it each hold a key whose exact score
 //      is at least lowS = m_k - err(m_k), so the true k-th best score t_k is at least lowS, and a group
 //      whose maximum g satisfies g + err(g) < lowS cannot hold one of the k best keys: it is skipped.
 //      err(T) = a + r |T| bounds |fp16 score - exact scaled score| (f16_filter.cuh).
@@ -14,11 +14,12 @@
 //      still hold a better key: the row goes to the redo list and the exact CUDA-core kernel
 //      recomputes it from all keys.  That needs more than L groups within the error bound of the
 //      k-th best score, which well-separated scores never produce; rows whose keys tie massively do.
-// One warp per (query, head); one candidate key per lane and step.
+// One warp per (query, head); a candidate key's row is read by D / 8 neighbouring lanes.
 #include <algorithm>
 
 #include "common.cuh"
 #include "f16_filter.cuh"
+#include "ptx.cuh"
 #include "topk_buffer.cuh"
 
 #include <cuda_fp16.h>
@@ -40,8 +41,12 @@ __device__ inline int graph_end_of(const int32_t* offs, int G, int N, int i) {
     return max(0, min(N, __ldg(offs + a + 1)));
 }
 
+// fp16 bits -> 16-bit key whose unsigned order is the order of the values (no NaNs reach this point)
+__device__ __forceinline__ unsigned f16_ordered(unsigned hb) { return (hb & 0x8000u) ? (~hb & 0xFFFFu) : (hb | 0x8000u); }
+__device__ __forceinline__ unsigned f16_unordered(unsigned ok) { return (ok & 0x8000u) ? (ok & 0x7FFFu) : (~ok & 0xFFFFu); }
+
 template <int D, int E, int LIST>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 4)
 refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                   const int32_t* __restrict__ offs, int G, int N, int H, int k,
                   const uint32_t* __restrict__ cand_word, const uint16_t* __restrict__ cand_half,
@@ -54,55 +59,74 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
     constexpr int KSTEPS = D / 16;
     static_assert(E <= 4 && LIST <= 64 && D <= 32, "k <= 32, head widths 16 and 32");
     __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
-    __shared__ float s_q[kWarpsPerBlock][D];
+    __shared__ __align__(16) float s_q[kWarpsPerBlock][D];
     __shared__ uint32_t s_words[kWarpsPerBlock][LIST];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     cand_t* row = s_rows[wib];
     float* q = s_q[wib];
     uint32_t* words = s_words[wib];
     const long long n_rows = (long long)N * H;
+    const long long stride = (long long)gridDim.x * kWarpsPerBlock;
     const int room = CAP - k;
+    constexpr int P = D / 8;                   // 16-byte pieces of a key row
+    constexpr int kRowStride = D * 2 + 16;     // padded: a lane per row reads 16-byte pieces without bank conflicts
+    constexpr int kStageBytes = 32 * kRowStride;
+    extern __shared__ __align__(16) unsigned char s_stage[];  // [warp][2 stages][32 rows]
+    unsigned char* stage = s_stage + wib * 2 * kStageBytes;
+    const int pl = lane % P;
+    const unsigned row_bytes = (unsigned)(H * D * (int)sizeof(T));
 
-    for (long long r = (long long)blockIdx.x * kWarpsPerBlock + wib; r < n_rows;
-         r += (long long)gridDim.x * kWarpsPerBlock) {
-        const int i = (int)(r / H), h = (int)(r % H);
-        const int hi = graph_end_of(offs, G, N, i);
-
-        // the row's groups: entry t in lane t%32, register t/32
-        uint32_t word[EPL];
-        float g[EPL];
-        bool valid[EPL];
-        int n_valid = 0;
+    // a row's list (entry t in lane t % 32, register t / 32) and query element are fetched one row ahead
+    uint32_t nx_word[EPL];
+    unsigned nx_half[EPL];
+    float nx_q = 0.0f;
+    auto fetch = [&](long long r) {
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int t = e * 32 + lane;
-            word[e] = 0u;
-            g[e] = -CUDART_INF_F;
-            valid[e] = false;
-            if (t < LIST) {
-                const unsigned short hb = __ldg(cand_half + (size_t)r * LIST + t);
-                // empty slots: the four-pipeline sweep marks them by the half 0xFFFF and never writes their
-                // group word, the ring sweep writes an all-ones word
-                if (hb != 0xFFFFu) {
-                    word[e] = __ldg(cand_word + (size_t)r * LIST + t);
-                    valid[e] = word[e] != 0xFFFFFFFFu;
-                    if (valid[e]) g[e] = __half2float(__ushort_as_half(hb));
-                }
+            nx_half[e] = 0xFFFFu;
+            nx_word[e] = 0xFFFFFFFFu;
+            if (r < n_rows && t < LIST) {
+                nx_half[e] = __ldg(cand_half + (size_t)r * LIST + t);
+                nx_word[e] = __ldg(cand_word + (size_t)r * LIST + t);  // never written for an empty slot: ignored below
             }
-            n_valid += __popc(__ballot_sync(FULL, valid[e]));
         }
+        nx_q = (r < n_rows && lane < D) ? Elem<T>::load(Q + (size_t)r * D + lane) : 0.0f;
+    };
+    long long r = (long long)blockIdx.x * kWarpsPerBlock + wib;
+    fetch(r);
 
-        // the query row and its norms; error bound of the fp16 scores in the scaled units of the sweep
+    for (; r < n_rows; r += stride) {
+        const int i = (int)(r / H), h = (int)(r % H);
+        const int hi = graph_end_of(offs, G, N, i);
+
+        // empty slots: the four-pipeline sweep marks them by the half 0xFFFF and never writes their group word,
+        // the ring sweep writes an all-ones word
+        uint32_t word[EPL];
+        unsigned okey[EPL];  // ordered 16-bit key of the group maximum; 0 for an empty slot (below every value)
+        int n_valid = 0;
+        unsigned ok_min = 0xFFFFu;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            word[e] = nx_word[e];
+            const bool valid = nx_half[e] != 0xFFFFu && word[e] != 0xFFFFFFFFu;
+            okey[e] = valid ? f16_ordered(nx_half[e]) : 0u;
+            n_valid += __popc(__ballot_sync(FULL, valid));
+            ok_min = min(ok_min, valid ? okey[e] : 0xFFFFu);
+        }
+        const float qc = nx_q;
         __syncwarp();
-        float qc = 0.0f;
-        if (lane < D) qc = Elem<T>::load(Q + (size_t)r * D + lane);
         if (lane < D) q[lane] = qc;
         for (int t = lane; t < k; t += 32) row[t] = 0ull;
+        fetch(r + stride);
+
+        // the query's norms; error bound of the fp16 scores in the scaled units of the sweep
         float q2 = qc * qc, qa2 = lane < 16 ? qc * qc : 0.0f;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             q2 += __shfl_xor_sync(FULL, q2, o);
             qa2 += __shfl_xor_sync(FULL, qa2, o);
+            ok_min = min(ok_min, __shfl_xor_sync(FULL, ok_min, o));
         }
         const F16HeadStat hs = stat[h];
         const float sq = f16_scale_from_n2max(hs.q_n2max), sk = f16_scale_from_n2max(hs.k_n2max);
@@ -112,36 +136,21 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
         const float ea = f16_abs_err(KSTEPS, nqa, nka, nq, nk) * 1.0001f;
         const float er = kF16RelErr;
         const float fp32_err = 4e-6f * nq * nk;  // of the fp32 rescoring below, in scaled units
-        __syncwarp();
+        const float g_min = __half2float(__ushort_as_half((unsigned short)f16_unordered(ok_min)));
 
-        // m_k: the entry that k-1 entries beat (value desc, slot asc)
+        // m_k, the k-th largest group maximum: the largest 16-bit key that at least k entries reach, bit by bit
         float lowS = -CUDART_INF_F;
-        float g_min = CUDART_INF_F;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) g_min = fminf(g_min, valid[e] ? g[e] : CUDART_INF_F);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) g_min = fminf(g_min, __shfl_xor_sync(FULL, g_min, o));
         if (n_valid >= k) {
-            int rank[EPL];
+            unsigned v = 0u;
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) rank[e] = 0;
+            for (int bit = 15; bit >= 0; --bit) {
+                const unsigned c = v | (1u << bit);
+                int n = 0;
 #pragma unroll
-            for (int e2 = 0; e2 < EPL; ++e2) {
-#pragma unroll 8
-                for (int l = 0; l < 32; ++l) {
-                    const float og = __shfl_sync(FULL, g[e2], l);
-                    const int ot = e2 * 32 + l;
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e)
-                        rank[e] += (og > g[e] || (og == g[e] && ot < e * 32 + lane)) ? 1 : 0;
-                }
+                for (int e = 0; e < EPL; ++e) n += __popc(__ballot_sync(FULL, okey[e] >= c));
+                if (n >= k) v = c;
             }
-            float mk = -CUDART_INF_F;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e)
-                if (valid[e] && rank[e] == k - 1) mk = g[e];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mk = fmaxf(mk, __shfl_xor_sync(FULL, mk, o));
+            const float mk = __half2float(__ushort_as_half((unsigned short)f16_unordered(v)));
             lowS = mk - ea - er * fabsf(mk);
         }
 
@@ -149,7 +158,8 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
         int n_kept = 0;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
-            const bool keep = valid[e] && (g[e] + ea + er * fabsf(g[e]) >= lowS);
+            const float g = __half2float(__ushort_as_half((unsigned short)f16_unordered(okey[e])));
+            const bool keep = okey[e] != 0u && (g + ea + er * fabsf(g) >= lowS);
             const unsigned m = __ballot_sync(FULL, keep);
             if (keep) words[n_kept + __popc(m & ((1u << lane) - 1u))] = word[e];
             n_kept += __popc(m);
@@ -160,50 +170,70 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
         const float floor_tau = n_valid >= k ? (lowS - fp32_err) / sc - 1e-30f : -CUDART_INF_F;
         float tau = floor_tau;
         int cnt = 0;
-        constexpr int NV = D * 2 / 16;  // 16-byte vectors per key row
-        constexpr int U = 2;            // steps whose loads are issued together
-        for (int t0 = 0; t0 < n_kept; t0 += U * 4) {
-            int jj[U];
-            bool kv[U];
-            uint4 raw[U][NV];
+        // Rescoring, 32 keys (4 groups) per step.  A key row is P = D / 8 pieces of 16 bytes.  The rows come in by
+        // asynchronous 16-byte copies in which P neighbouring lanes fetch one row, so one copy instruction touches
+        // 32 / P cache lines instead of 32 (the kernel is bound by these line accesses); they land in a per-warp
+        // stage of padded rows, one step ahead of the arithmetic.  Then each lane reads one whole row back and
+        // scores it with the same chain of fused multiply-adds in index order as every other kernel.
+        const int nsteps = (n_kept + 3) / 4;
+        const unsigned char* kb = reinterpret_cast<const unsigned char*>(K) + ((size_t)h * D + pl * 8) * sizeof(T);
+        auto issue = [&](int step) {
+            if (step < nsteps) {
+                unsigned char* buf = stage + (step & 1) * kStageBytes;
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int t = t0 + u * 4 + (lane >> 3);
-                const uint32_t wd = t < n_kept ? words[t] : 0u;
-                jj[u] = (int)(wd & 0x7FFFFFFFu) + (int)(wd >> 31) + 2 * (lane & 7);
-                kv[u] = t < n_kept && jj[u] < hi && kmip_check(jj[u] >= 0 && hi <= N, sb, 101);  // checks builds: key row inside K
-                if (kv[u]) {
-                    const uint4* kr = reinterpret_cast<const uint4*>(K + ((size_t)jj[u] * H + h) * D);
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) raw[u][v] = __ldg(kr + v);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                float s = 0.0f;
-                if (kv[u]) {
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        const uint32_t wv[4] = {raw[u][v].x, raw[u][v].y, raw[u][v].z, raw[u][v].w};
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) {
-                            s = fmaf(q[v * 8 + 2 * x], __uint_as_float(wv[x] << 16), s);
-                            s = fmaf(q[v * 8 + 2 * x + 1], __uint_as_float(wv[x] & 0xFFFF0000u), s);
-                        }
-                    }
-                }
-                const bool pass = kv[u] && (s > tau);
-                const unsigned m = __ballot_sync(FULL, pass);
-                if (m) {
-                    if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, jj[u]);
-                    cnt += __popc(m);
-                    if (cnt > room - 32) {
-                        tau = fmaxf(floor_tau, warp_merge_row_chunks(row, k, cnt, lane));
-                        cnt = 0;
+                for (int c = 0; c < P; ++c) {  // copy instruction c: keys c * 32 / P ... of the step
+                    const int rrow = c * (32 / P) + lane / P;  // row of the stage = key of the step
+                    const int t = step * 4 + (rrow >> 3);
+                    if (t < n_kept) {
+                        const uint32_t wd = words[t];
+                        const int j = (int)(wd & 0x7FFFFFFFu) + (int)(wd >> 31) + 2 * (rrow & 7);
+                        if (j < hi && kmip_check(j >= 0 && hi <= N, sb, 101))  // checks builds: key row inside K
+                            ptx::cp_async_16(buf + rrow * kRowStride + pl * 16, kb + (size_t)(unsigned)j * row_bytes);
                     }
                 }
             }
+            ptx::cp_async_commit();  // an empty group when there is nothing left, so that the count below holds
+        };
+        issue(0);
+        for (int step = 0; step < nsteps; ++step) {
+            issue(step + 1);
+            ptx::cp_async_wait<1>();  // all but the newest group: this step's rows are in
+            __syncwarp();
+            const int t = step * 4 + (lane >> 3);
+            const uint32_t wd = t < n_kept ? words[t] : 0u;
+            const int jj = (int)(wd & 0x7FFFFFFFu) + (int)(wd >> 31) + 2 * (lane & 7);
+            const bool kv = t < n_kept && jj < hi;
+            float s = 0.0f;
+            if (kv) {
+                const unsigned char* kr = stage + (step & 1) * kStageBytes + lane * kRowStride;
+#pragma unroll
+                for (int v = 0; v < P; ++v) {
+                    const uint4 rw = *reinterpret_cast<const uint4*>(kr + v * 16);
+                    const uint32_t wv[4] = {rw.x, rw.y, rw.z, rw.w};
+                    const float4 qa = *reinterpret_cast<const float4*>(q + v * 8), qb = *reinterpret_cast<const float4*>(q + v * 8 + 4);
+                    const float qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        s = fmaf(qv[2 * x], __uint_as_float(wv[x] << 16), s);
+                        s = fmaf(qv[2 * x + 1], __uint_as_float(wv[x] & 0xFFFF0000u), s);
+                    }
+                }
+            }
+            const bool pass = kv && (s > tau);
+            const unsigned m = __ballot_sync(FULL, pass);
+            if (m) {
+                if (pass) row[k + cnt + __popc(m & ((1u << lane) - 1u))] = make_cand(s, jj);
+                cnt += __popc(m);
+                if (cnt > room - 32) {
+                    // the groups come in list order, not key order: a later key with the same score as the
+                    // k-th best and a smaller index must still get in, so the threshold sits just below it
+                    tau = fmaxf(floor_tau, nextafterf(warp_merge_row_chunks(row, k, cnt, lane), -CUDART_INF_F));
+                    cnt = 0;
+                }
+            }
+            __syncwarp();  // the stage is free for the copies of step + 2
         }
+        ptx::cp_async_wait<0>();
         const float kth = warp_merge_row_chunks(row, k, cnt, lane);
         // a dropped group scores at most g_min + err(g_min) exactly (scaled); it matters if that reaches the
         // k-th best score found
@@ -214,6 +244,7 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
             }
         }
         warp_store_row(row, k, lane, topk_idx + (size_t)r * k, topk_score + (size_t)r * k);
+        __syncwarp();
     }
 }
 
@@ -221,16 +252,19 @@ template <int D>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w) {
     const long long n_rows = (long long)a.N * a.H;
     const int blocks = (int)std::min<long long>((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock, (long long)sm_count() * 32);
+    constexpr int kSmem = kWarpsPerBlock * 2 * 32 * (D * 2 + 16);  // the rescoring stages
 #define KMIP_LAUNCH_REFINE16(E_, LIST_) \
-    refine_f16_kernel<D, E_, LIST_><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>( \
+    if ((err = cudaFuncSetAttribute(refine_f16_kernel<D, E_, LIST_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem)) != cudaSuccess) return err; \
+    refine_f16_kernel<D, E_, LIST_><<<blocks, kWarpsPerBlock * 32, kSmem, a.stream>>>( \
         static_cast<const __nv_bfloat16*>(a.Q), static_cast<const __nv_bfloat16*>(a.K), a.graph_offsets, a.G, (int)a.N, \
         a.H, a.k, reinterpret_cast<const uint32_t*>(a.ws + w.cand_word_off), \
         reinterpret_cast<const uint16_t*>(a.ws + w.cand_half_off), reinterpret_cast<const F16HeadStat*>(a.ws + w.f16stat_off), \
         a.topk_idx, a.topk_score, reinterpret_cast<StatusBlock*>(a.ws), reinterpret_cast<int*>(a.ws + w.redo_off))
+    cudaError_t err;
     // the list sizes are those of score_select_f16_list
-    if (a.k <= 8) KMIP_LAUNCH_REFINE16(2, 16);
-    else if (a.k <= 16) KMIP_LAUNCH_REFINE16(2, 24);
-    else KMIP_LAUNCH_REFINE16(4, 48);
+    if (a.k <= 8) { KMIP_LAUNCH_REFINE16(2, 16); }
+    else if (a.k <= 16) { KMIP_LAUNCH_REFINE16(2, 24); }
+    else { KMIP_LAUNCH_REFINE16(4, 48); }
 #undef KMIP_LAUNCH_REFINE16
     return cudaGetLastError();
 }
