@@ -230,126 +230,176 @@ scan_inplace_kernel(int* __restrict__ v, long long n, const int* __restrict__ bl
 
 // ---- hit lists by a stable radix sort --------------------------------------------------------------
 // A hit record is everything the segment reduction needs about one selected pair in one 16-byte load:
-// {query row, softmax weight p (times the dropout factor), score gradient dS, (key, head) number}.  The
+// {query row, softmax weight p (times the dropout factor), score gradient dS, (key, head) number}.
 // The records are sorted by (key, head) number in two stable steps, and the pairs start out in query
 // order, so each key's list ends up ordered by query row - the same order on every run, which makes the
 // sums of the segment stage reproducible bit for bit.  Pairs without a key (padding slots) get the number
 // n_rows and sort behind every list.
-//   partition  by the high digit of the number into buckets of 2^lo consecutive numbers: kRadixSlots warps
-//              own contiguous ranges of the pairs; each counts the digits of its range, an exclusive scan
-//              over (digit, slot) turns the counts into start offsets, and each warp walks its range again,
-//              32 records at a time, ranks equal digits by lane with a match vote and advances its own
-//              offsets - no atomics, so nothing depends on timing.  This is the one pass that scatters
-//              16-byte records over the whole buffer.
+//   partition  by the high digit of the number into buckets of 2^lo consecutive numbers.  A block owns a
+//              contiguous range of the pairs (512 per warp).  A first kernel counts the digits of every block;
+//              an exclusive scan over (digit, block) gives every block the place where its records of a digit
+//              start.  The second kernel sorts the block's records by digit inside shared memory - each warp
+//              counts the digits of its part, the counts are prefix-summed over the warps and the digits,
+//              and each warp walks its part again, 32 records at a time, ranking equal digits by lane with a
+//              match vote and advancing its own offsets - and then copies the sorted block out, so that the
+//              records of a digit leave as one contiguous run.  No atomics decide a position: nothing depends
+//              on timing.
 //   buckets    one block per bucket sorts its records (a few hundred KB, served by L2) by the low digit
 //              with the same count / scan / ranked walk, its eight warps owning contiguous parts.
 struct RadixSrc {
-    const int32_t* topk_idx;  // first pass: the records are built from the pairs
+    const int32_t* topk_idx;
     const float* ws_p;
     const float* ws_ds;
-    const int4* recs;         // later passes
     int N, H, k;
     int n_rows;
 };
 
-template <bool FIRST>
-__device__ __forceinline__ int4 radix_load(const RadixSrc& s, long long e) {
-    if (!FIRST) return __ldg(s.recs + e);
-    const int j = __ldg(s.topk_idx + e);
-    const long long r = e / s.k;  // query * H + head
-    const int key = (j >= 0 && j < s.N) ? j * s.H + (int)(r % s.H) : s.n_rows;
-    return make_int4((int)(r / s.H), __float_as_int(__ldg(s.ws_p + e)), __float_as_int(__ldg(s.ws_ds + e)), key);
+// Lanes of the warp whose digit equals this lane's; lanes that hold no record vote with values of their own,
+// which match nobody.
+__device__ __forceinline__ unsigned warp_same_digit(int digit, bool live) {
+    return __match_any_sync(0xFFFFFFFFu, live ? digit : (1 << kRadixMaxBits) + (int)(threadIdx.x & 31));
 }
 
-// Per-warp digit counters are 16 bits wide (a warp's range holds fewer than 65536 records), two to a word.
-template <bool FIRST>
-__global__ void __launch_bounds__(kRadixWarps * 32)
-radix_count_kernel(const RadixSrc src, long long n, long long per_slot, int shift, int bins, int* __restrict__ table,
-                   StatusBlock* __restrict__ sb) {
-    extern __shared__ unsigned s_hist[];  // [kRadixWarps][bins / 2]
-    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int words = bins / 2;
-    for (int x = threadIdx.x; x < kRadixWarps * words; x += blockDim.x) s_hist[x] = 0u;
-    __syncthreads();
-    const int slot = blockIdx.x * kRadixWarps + w;
-    const long long lo = (long long)slot * per_slot, hi = min(n, lo + per_slot);
-    unsigned* hist = s_hist + w * words;
-    constexpr int U = 8;  // loads in flight per lane
-    for (long long e0 = lo; e0 < hi; e0 += 32 * U) {
-        int key[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long long e = e0 + u * 32 + lane;
-            key[u] = -1;
-            if (e < hi) {
-                if (FIRST) {
-                    const int j = __ldg(src.topk_idx + e);
-                    kmip_check(j < src.N, sb, 105);  // checks builds: an index the forward pass cannot have written (ignored either way)
-                    key[u] = (j >= 0 && j < src.N) ? j * src.H + (int)((e / src.k) % src.H) : src.n_rows;
-                } else {
-                    key[u] = __ldg(reinterpret_cast<const int*>(src.recs + e) + 3);
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (key[u] >= 0) {
-                const int d = (key[u] >> shift) & (bins - 1);
-                atomicAdd(hist + (d >> 1), 1u << (16 * (d & 1)));  // shared memory; the counts do not depend on the order
-            }
-        }
-    }
-    __syncthreads();
-    for (int x = threadIdx.x; x < kRadixWarps * bins; x += blockDim.x) {
-        const int ww = x / bins, d = x % bins;
-        table[(size_t)d * kRadixSlots + blockIdx.x * kRadixWarps + ww] = (int)((s_hist[ww * words + (d >> 1)] >> (16 * (d & 1))) & 0xFFFFu);
-    }
+__device__ __forceinline__ int radix_key(const RadixSrc& s, long long e, int j) {
+    return (j >= 0 && j < s.N) ? j * s.H + (int)((e / s.k) % s.H) : s.n_rows;
 }
 
-template <bool FIRST>
-__global__ void __launch_bounds__(kRadixWarps * 32)
-radix_scatter_kernel(const RadixSrc src, long long n, long long per_slot, int shift, int bins, const int* __restrict__ table,
+// table[digit][block] = number of the block's pairs with that high digit
+__global__ void __launch_bounds__(512)
+radix_count_kernel(const RadixSrc src, long long n, int per_block, int shift, int bins, int n_blocks,
+                   int* __restrict__ table, StatusBlock* __restrict__ sb) {
+    extern __shared__ unsigned s_hist[];  // [bins]
+    for (int x = threadIdx.x; x < bins; x += blockDim.x) s_hist[x] = 0u;
+    __syncthreads();
+    const long long lo = (long long)blockIdx.x * per_block, hi = min(n, lo + per_block);
+    for (long long e = lo + threadIdx.x; e < hi; e += blockDim.x) {
+        const int j = __ldg(src.topk_idx + e);
+        kmip_check(j < src.N, sb, 105);  // checks builds: an index the forward pass cannot have written (ignored either way)
+        atomicAdd(s_hist + ((radix_key(src, e, j) >> shift) & (bins - 1)), 1u);  // shared memory; the counts do not depend on the order
+    }
+    __syncthreads();
+    for (int d = threadIdx.x; d < bins; d += blockDim.x) table[(size_t)d * n_blocks + blockIdx.x] = (int)s_hist[d];
+}
+
+// table: after the scan, table[digit][block] is where the block's records of that digit start in dst.
+// Shared memory: the block's records [warps * 512] (16 bytes each), per-warp digit counters (16 bits, [warps][bins]),
+// where each digit starts inside the block (16 bits, [bins]) and in dst (32 bits, [bins]).
+__global__ void __launch_bounds__(512)
+radix_scatter_kernel(const RadixSrc src, long long n, int shift, int bins, int n_blocks, const int* __restrict__ table,
                      int4* __restrict__ dst, StatusBlock* __restrict__ sb) {
-    extern __shared__ unsigned s_hist[];  // viewed as unsigned short [kRadixWarps][bins]: records of each digit placed so far
-    unsigned short* s_cnt = reinterpret_cast<unsigned short*>(s_hist);
+    extern __shared__ int4 s_rec[];
+    const int warps = blockDim.x >> 5, per_block = warps * kRadixPerWarp;
+    unsigned short* s_cnt = reinterpret_cast<unsigned short*>(s_rec + per_block);
+    unsigned short* s_dstart = s_cnt + warps * bins;
+    int* s_base = reinterpret_cast<int*>(s_dstart + bins);
+    __shared__ int s_scan[16];
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int x = threadIdx.x; x < kRadixWarps * bins / 2; x += blockDim.x) s_hist[x] = 0u;
+    for (int x = threadIdx.x; x < warps * bins / 2; x += blockDim.x) reinterpret_cast<unsigned*>(s_cnt)[x] = 0u;
+    for (int d = threadIdx.x; d < bins; d += blockDim.x) s_base[d] = __ldg(table + (size_t)d * n_blocks + blockIdx.x);
     __syncthreads();
-    const int slot = blockIdx.x * kRadixWarps + w;
-    const long long lo = (long long)slot * per_slot, hi = min(n, lo + per_slot);
+    const long long lo = (long long)blockIdx.x * per_block + (long long)w * kRadixPerWarp;
+    const long long hi = min(n, lo + kRadixPerWarp);
+    constexpr int R = kRadixPerWarp / 32;  // rounds of 32 pairs per warp
+    int key[R];
+    float pw[R], dsw[R];  // everything the block reads from memory is requested here, before any of it is used
     unsigned short* cnt = s_cnt + w * bins;
-    const int* start = table + slot;  // start[d * kRadixSlots]: where this warp's records of digit d begin
+#pragma unroll
+    for (int u = 0; u < R; ++u) {
+        const long long e = lo + u * 32 + lane;
+        key[u] = e < hi ? __ldg(src.topk_idx + e) : -1;
+        pw[u] = e < hi ? __ldg(src.ws_p + e) : 0.0f;
+        dsw[u] = e < hi ? __ldg(src.ws_ds + e) : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < R; ++u) {
+        const long long e = lo + u * 32 + lane;
+        key[u] = e < hi ? radix_key(src, e, key[u]) : -1;
+    }
+    // the warp's digit counts (two 16-bit counters to a word; shared-memory atomics: counts do not depend on the order)
     const unsigned lt = (1u << lane) - 1u;
-    constexpr int U = 8;  // records loaded ahead per lane; they are placed in order, 32 at a time
-    for (long long e0 = lo; e0 < hi; e0 += 32 * U) {
-        int4 recs[U];
-        int base[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const long long e = e0 + u * 32 + lane;
-            recs[u] = make_int4(0, 0, 0, -1);
-            if (e < hi) recs[u] = radix_load<FIRST>(src, e);
+    for (int u = 0; u < R; ++u) {
+        if (key[u] >= 0) {
+            const int digit = (key[u] >> shift) & (bins - 1);
+            atomicAdd(reinterpret_cast<unsigned*>(cnt) + (digit >> 1), 1u << (16 * (digit & 1)));
         }
+    }
+    __syncthreads();
+    // counts -> offsets: per digit over the warps, then over the digits (each thread owns DPT consecutive digits)
+    {
+        const int DPT = (bins + (int)blockDim.x - 1) / (int)blockDim.x;
+        const int d0 = threadIdx.x * DPT;
+        int mine = 0;
+        for (int i = 0; i < DPT; ++i) {
+            const int d = d0 + i;
+            if (d >= bins) break;
+            int c[16];
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-            base[u] = recs[u].w >= 0 ? __ldg(start + (size_t)((recs[u].w >> shift) & (bins - 1)) * kRadixSlots) : 0;
+            for (int ww = 0; ww < 16; ++ww) c[ww] = ww < warps ? s_cnt[ww * bins + d] : 0;
+            int run = 0;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (e0 + u * 32 >= hi) break;  // warp-uniform
-            const int4 rec = recs[u];
-            const bool live = e0 + u * 32 + lane < hi;
-            // lanes past the end of the range vote with digits of their own, which match nobody
-            const int digit = live ? ((rec.w >> shift) & (bins - 1)) : bins + lane;
-            const unsigned same = __match_any_sync(0xFFFFFFFFu, digit);
-            if (live) {
-                const int placed = cnt[digit];
-                const long long pos = (long long)base[u] + placed + __popc(same & lt);
-                if (kmip_check(pos >= 0 && pos < n, sb, 104)) dst[pos] = rec;  // checks builds: inside the buffer
-                __syncwarp(same);
-                if ((same & lt) == 0u) cnt[digit] = (unsigned short)(placed + __popc(same));  // the group's first lane moves the digit on
+            for (int ww = 0; ww < 16; ++ww) {
+                if (ww < warps) s_cnt[ww * bins + d] = (unsigned short)run;
+                run += c[ww];
             }
-            __syncwarp();
+            s_dstart[d] = (unsigned short)run;  // the digit's total for now
+            mine += run;
         }
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_scan[w] = incl;
+        __syncthreads();
+        if (w == 0) {
+            int v = lane < warps ? s_scan[lane] : 0;
+#pragma unroll
+            for (int o = 1; o < 16; o <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, v, o);
+                if (lane >= o) v += t;
+            }
+            if (lane < warps) s_scan[lane] = v;
+        }
+        __syncthreads();
+        int run = (w ? s_scan[w - 1] : 0) + incl - mine;
+        for (int i = 0; i < DPT; ++i) {
+            const int d = d0 + i;
+            if (d >= bins) break;
+            const int c = s_dstart[d];
+            s_dstart[d] = (unsigned short)run;
+            run += c;
+        }
+    }
+    __syncthreads();
+    // ranked walk into the block's sorted order
+#pragma unroll
+    for (int u = 0; u < R; ++u) {
+        const long long e = lo + u * 32 + lane;
+        const bool live = key[u] >= 0;
+        int4 rec = make_int4(0, 0, 0, 0);
+        if (live) {
+            const long long r = e / src.k;  // query * H + head
+            rec = make_int4((int)(r / src.H), __float_as_int(pw[u]), __float_as_int(dsw[u]), key[u]);
+        }
+        const int digit = (key[u] >> shift) & (bins - 1);
+        const unsigned same = warp_same_digit(digit, live);
+        if (live) {
+            const int placed = cnt[digit];
+            s_rec[s_dstart[digit] + placed + __popc(same & lt)] = rec;
+            __syncwarp(same);
+            if ((same & lt) == 0u) cnt[digit] = (unsigned short)(placed + __popc(same));  // the group's first lane moves the digit on
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+    const int total = (int)min((long long)per_block, n - (long long)blockIdx.x * per_block);
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const int4 rec = s_rec[i];
+        const int digit = (rec.w >> shift) & (bins - 1);
+        const long long pos = (long long)s_base[digit] + (i - (int)s_dstart[digit]);
+        if (kmip_check(pos >= 0 && pos < n, sb, 104)) dst[pos] = rec;  // checks builds: inside the buffer
     }
 }
 
@@ -372,12 +422,12 @@ __global__ void fill_unordered_kernel(const int32_t* __restrict__ topk_idx, long
 }
 
 // Second step: the records of one bucket (high digit = blockIdx.x), src -> dst, ordered by the low digit and,
-// within a digit, in the order they have in src.  bucket_start[d * kRadixSlots] is where bucket d begins.  The low
+// within a digit, in the order they have in src.  bucket_start[d * start_stride] is where bucket d begins.  The low
 // digit of a number inside its bucket IS the (key, head) pair, so this kernel also knows where every list starts:
 // it writes seg_off (rows + 1 entries) and the list of long segments.
 constexpr int kBucketWarps = 8;
 __global__ void __launch_bounds__(kBucketWarps * 32)
-radix_bucket_kernel(const int4* __restrict__ src, int4* __restrict__ dst, const int* __restrict__ bucket_start, int n_buckets,
+radix_bucket_kernel(const int4* __restrict__ src, int4* __restrict__ dst, const int* __restrict__ bucket_start, int start_stride, int n_buckets,
                     long long n, int lo_bits, long long n_rows, int* __restrict__ seg_off, int* __restrict__ long_list,
                     StatusBlock* __restrict__ sb) {
     extern __shared__ int s_cnt[];  // [kBucketWarps][bins]: counts, then next free positions
@@ -386,8 +436,8 @@ radix_bucket_kernel(const int4* __restrict__ src, int4* __restrict__ dst, const 
     const int bins = 1 << lo_bits;
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int d_hi = blockIdx.x;
-    const long long begin = bucket_start[(size_t)d_hi * kRadixSlots];
-    const long long end = d_hi + 1 < n_buckets ? (long long)bucket_start[(size_t)(d_hi + 1) * kRadixSlots] : n;
+    const long long begin = bucket_start[(size_t)d_hi * start_stride];
+    const long long end = d_hi + 1 < n_buckets ? (long long)bucket_start[(size_t)(d_hi + 1) * start_stride] : n;
     const long long len = end - begin;
     for (int x = threadIdx.x; x < kBucketWarps * bins; x += blockDim.x) s_cnt[x] = 0;
     if (threadIdx.x == 0) s_carry = 0;
@@ -465,8 +515,8 @@ radix_bucket_kernel(const int4* __restrict__ src, int4* __restrict__ dst, const 
             if (e0 + u * 32 >= hi) break;  // warp-uniform
             const int4 rec = recs[u];
             const bool live = e0 + u * 32 + lane < hi;
-            const int digit = live ? (rec.w & (bins - 1)) : bins + lane;
-            const unsigned same = __match_any_sync(0xFFFFFFFFu, digit);
+            const int digit = rec.w & (bins - 1);
+            const unsigned same = warp_same_digit(digit, live);
             if (live) {
                 const int base = cnt[digit];
                 const long long pos = begin + base + __popc(same & lt);
@@ -653,11 +703,9 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
     // the hit lists: stable partition of the pairs by the high digit of their (key, head) number, then a stable
     // sort of every bucket by the low digit, which also writes the list offsets
     {
-        int bits, lo_bits, hi_bits;
-        radix_digits(n_rows, bits, lo_bits, hi_bits);
-        const long long per_slot = ((n_pairs + kRadixSlots - 1) / kRadixSlots + 31) / 32 * 32;
-        if (bits > 2 * kRadixMaxBits || per_slot > 65535) {
-            // more than 16.7 million (node, head) pairs or 465 million selected pairs: unordered lists
+        const RadixPlan rp = plan_radix(n_rows, n_pairs);
+        if (!rp.sorted) {
+            // more than 16.7 million (node, head) pairs or 2^31 selected pairs: unordered lists
             if ((err = cudaMemsetAsync(cursor, 0, sizeof(int) * (size_t)(n_rows + 1), a.stream)) != cudaSuccess) return err;
             hist_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, cursor, sb);
             scan_block_sums_kernel<<<w.scan_blocks, kScanThreads, 0, a.stream>>>(cursor, n_rows, block_sums);
@@ -666,21 +714,23 @@ cudaError_t launch_d(const BwdArgs& a, const BwdWorkspace& w, cudaEvent_t* ev) {
             fill_unordered_kernel<<<pair_blocks, 256, 0, a.stream>>>(a.topk_idx, n_pairs, (int)a.N, a.H, a.k, ws_p, ws_ds, seg_off,
                                                                     cursor, hits, sb);
         } else {
-            const int bins_hi = 1 << hi_bits, bins_lo = 1 << lo_bits;
-            const long long n_tab = (long long)bins_hi * kRadixSlots;
+            const int bins_hi = 1 << rp.hi_bits, bins_lo = 1 << rp.lo_bits, n_blocks = (int)rp.blocks;
+            const int per_block = rp.warps * kRadixPerWarp;
+            const long long n_tab = (long long)bins_hi * n_blocks;
             const int tab_blocks = (int)((n_tab + kScanItemsPerBlock - 1) / kScanItemsPerBlock);
-            const size_t smem_hi = (size_t)kRadixWarps * bins_hi * 2, smem_lo = (size_t)kBucketWarps * bins_lo * sizeof(int);
-            if ((err = cudaFuncSetAttribute(radix_count_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hi)) != cudaSuccess ||
-                (err = cudaFuncSetAttribute(radix_scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_hi)) != cudaSuccess ||
+            const size_t smem_cnt = (size_t)bins_hi * sizeof(unsigned);
+            const size_t smem_sct = (size_t)per_block * sizeof(int4) + (size_t)rp.warps * bins_hi * 2 + (size_t)bins_hi * 2 + (size_t)bins_hi * sizeof(int);
+            const size_t smem_lo = (size_t)kBucketWarps * bins_lo * sizeof(int);
+            if ((err = cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_sct)) != cudaSuccess ||
                 (err = cudaFuncSetAttribute(radix_bucket_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lo)) != cudaSuccess)
                 return err;
-            RadixSrc src{a.topk_idx, ws_p, ws_ds, nullptr, (int)a.N, a.H, a.k, (int)n_rows};
-            radix_count_kernel<true><<<kRadixBlocks, kRadixWarps * 32, smem_hi, a.stream>>>(src, n_pairs, per_slot, lo_bits, bins_hi, table, sb);
+            RadixSrc src{a.topk_idx, ws_p, ws_ds, (int)a.N, a.H, a.k, (int)n_rows};
+            radix_count_kernel<<<n_blocks, 512, smem_cnt, a.stream>>>(src, n_pairs, per_block, rp.lo_bits, bins_hi, n_blocks, table, sb);
             scan_block_sums_kernel<<<tab_blocks, kScanThreads, 0, a.stream>>>(table, n_tab, tblsum);
             scan_block_offsets_kernel<<<1, kScanThreads, 0, a.stream>>>(tblsum, tab_blocks);
             scan_inplace_kernel<<<tab_blocks, kScanThreads, 0, a.stream>>>(table, n_tab, tblsum);
-            radix_scatter_kernel<true><<<kRadixBlocks, kRadixWarps * 32, smem_hi, a.stream>>>(src, n_pairs, per_slot, lo_bits, bins_hi, table, tmp, sb);
-            radix_bucket_kernel<<<bins_hi, kBucketWarps * 32, smem_lo, a.stream>>>(tmp, hits, table, bins_hi, n_pairs, lo_bits, n_rows,
+            radix_scatter_kernel<<<n_blocks, rp.warps * 32, smem_sct, a.stream>>>(src, n_pairs, rp.lo_bits, bins_hi, n_blocks, table, tmp, sb);
+            radix_bucket_kernel<<<bins_hi, kBucketWarps * 32, smem_lo, a.stream>>>(tmp, hits, table, n_blocks, bins_hi, n_pairs, rp.lo_bits, n_rows,
                                                                                 seg_off, long_list, sb);
         }
     }

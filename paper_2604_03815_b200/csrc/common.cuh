@@ -154,7 +154,7 @@ struct BwdWorkspace {
     size_t cursor_off;    // int   [N*H]     hit counts, then fill cursors
     size_t pairs_off;     // int4  [N*H*k]   hit lists: records {query row, p, dS, (key, head) number}
     size_t tmp_off;       // int4  [N*H*k]   the other buffer of the radix passes that build them
-    size_t table_off;     // int   [high digits * kRadixSlots]  digit counts per (digit, slot), then offsets
+    size_t table_off;     // int   [high digits][blocks]  digit counts per block of the first sorting step, then offsets
     size_t tblsum_off;    // int   block sums of the scan over that table
     size_t blocksum_off;  // int   [scan blocks]
     size_t long_off;      // int   [N*H]     ids of long segments
@@ -164,17 +164,31 @@ struct BwdWorkspace {
 };
 
 constexpr int kScanItemsPerBlock = 4096;
-// The hit lists are built by a stable radix sort of the selected pairs by (key, head) number, so every list
-// comes out ordered by query row whatever the timing: kRadixSlots warps each own a contiguous range of pairs.
-constexpr int kRadixBlocks = 444, kRadixWarps = 16, kRadixSlots = kRadixBlocks * kRadixWarps;
+// The hit lists are built by a stable two-step radix sort of the selected pairs by (key, head) number, so every
+// list comes out ordered by query row whatever the timing.  First step: a block owns kRadixPerWarp consecutive
+// pairs per warp and sorts them by the high digit in shared memory before it writes them out.
+constexpr int kRadixPerWarp = 512;
 constexpr int kRadixMaxBits = 12, kRadixMaxBins = 1 << kRadixMaxBits;
-// digits of the two steps for `rows` (node, head) pairs: the numbers 0 .. rows (rows = "no key") split into a
-// high and a low digit; more than 2 * kRadixMaxBits bits are not sorted (unordered fallback)
-inline void radix_digits(long long rows, int& bits, int& lo_bits, int& hi_bits) {
-    bits = 1;
-    while ((1ll << bits) <= rows) ++bits;
-    lo_bits = bits / 2;
-    hi_bits = bits - lo_bits;
+struct RadixPlan {
+    int bits, lo_bits, hi_bits;  // of the numbers 0 .. rows (rows = "no key"): low and high digit
+    bool sorted;                 // false: more than 2 * kRadixMaxBits bits or 2^31 pairs, unordered lists instead
+    int warps;                   // per block of the first step
+    long long blocks;            // blocks of the first step
+    size_t bins_hi;
+};
+inline RadixPlan plan_radix(long long rows, long long pairs) {
+    RadixPlan r;
+    r.bits = 1;
+    while ((1ll << r.bits) <= rows) ++r.bits;
+    r.hi_bits = r.bits / 2 > 0 ? r.bits / 2 : 1;
+    r.lo_bits = r.bits - r.hi_bits;
+    r.sorted = r.bits <= 2 * kRadixMaxBits && pairs < (1ll << 31);
+    r.warps = 8;
+    const long long per_block = (long long)r.warps * kRadixPerWarp;
+    r.blocks = r.sorted ? (pairs + per_block - 1) / per_block : 1;
+    if (r.blocks < 1) r.blocks = 1;
+    r.bins_hi = r.sorted ? ((size_t)1 << r.hi_bits) : 1;
+    return r;
 }
 
 inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
@@ -193,11 +207,9 @@ inline BwdWorkspace plan_bwd_workspace(int64_t N, int32_t H, int32_t k) {
     w.cursor_off = o;   o = region(o + 4 * (rows + 1));
     w.pairs_off = o;    o = region(o + 16 * pairs);
     w.tmp_off = o;      o = region(o + 16 * pairs);
-    int bits, lo_bits, hi_bits;
-    radix_digits((long long)rows, bits, lo_bits, hi_bits);
-    const size_t bins_hi = bits <= 2 * kRadixMaxBits ? ((size_t)1 << hi_bits) : 1;
-    w.table_off = o;    o = region(o + 4 * bins_hi * kRadixSlots);
-    w.tblsum_off = o;   o = region(o + 4 * (bins_hi * kRadixSlots / kScanItemsPerBlock + 2));
+    const RadixPlan rp = plan_radix((long long)rows, (long long)pairs);
+    w.table_off = o;    o = region(o + 4 * rp.bins_hi * (size_t)rp.blocks);
+    w.tblsum_off = o;   o = region(o + 4 * (rp.bins_hi * (size_t)rp.blocks / kScanItemsPerBlock + 2));
     w.blocksum_off = o; o = region(o + 4 * (size_t)(w.scan_blocks + 1));
     w.long_off = o;     o = region(o + 4 * rows);
     w.total = o;
