@@ -79,7 +79,8 @@ typedef enum {
  * 32768 nodes on, one of Q in the sweep's row order plus 6 bytes per node
  * (tensor-core mode only), for head widths up to 32 and k <= 32 also 6 bytes per kept candidate group
  * (16, 24 or 48 per (node, head)), plus the work list; backward: 40 bytes per selected pair, 12 bytes per
- * (node, head) and a 39 MB table.  Host only, no CUDA call.
+ * (node, head) and a table of digit counts of the sort that builds the hit lists (at most 4 bytes per
+ * selected pair, 1 to 2 at the sizes of the paper's experiments).  Host only, no CUDA call.
  */
 int kmip_attn_workspace_bytes(int64_t N, int32_t G, int32_t H, int32_t d, int32_t k,
                               int mode, int pass, size_t *bytes);
@@ -120,8 +121,8 @@ int kmip_attn_forward(const void *Q, const void *K, const void *V,
  * arithmetic (indices are global) and may be NULL / 0.
  * dK and dV are sums over each key's list of hits in query order (the lists are built by a stable sort,
  * without atomics), so the same inputs give the same gradients bit for bit on every run (up to 2^24
- * (node, head) pairs; beyond that the lists are filled with atomic counters and the sums are
- * reproducible to fp32 rounding only).
+ * (node, head) pairs and 2^31 selected pairs; beyond that the lists are filled with atomic counters and
+ * the sums are reproducible to fp32 rounding only).
  */
 int kmip_attn_backward(const void *Q, const void *K, const void *V,
                        const int32_t *graph_offsets, int32_t G, int64_t N,

@@ -69,8 +69,8 @@ def test_workspace_bytes_host_only(kb):
     assert kb.kmip_attn_workspace_bytes(500_000, 1, 4, 32, 32, kb.KMIP_BF16_TC_PRUNED, kb.PASS_BACKWARD) == b
     pairs = 500_000 * 4 * 32
     # p, dS and two buffers of 16-byte hit records (the radix sort that orders them): 40 bytes per selected pair,
-    # 12 per (node, head), and a 39 MB table of digit counts
-    assert 40 * pairs < b < 40 * pairs + 14 * 500_000 * 4 + (40 << 20)
+    # 12 per (node, head), and the table of digit counts (1024 digits x 4 bytes per block of 4096 pairs)
+    assert 40 * pairs < b < 41 * pairs + 14 * 500_000 * 4 + (8 << 20)
     for bad in [dict(d=24), dict(k=129), dict(mode=7)]:
         args = dict(N=1000, G=1, H=2, d=32, k=8, mode=kb.KMIP_BF16_TC)
         args.update(bad)
