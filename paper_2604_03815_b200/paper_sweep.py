@@ -8,9 +8,9 @@ N = 10^(i/2).  The library stores head widths 16/32/64/128, so d_K = 10 is zero-
 
 --k changes the number of keys kept (the paper's appendix "Additional results", "Influence of k", reports
 whole-model epoch times for k up to 100, where its implementation slows down sharply).
-Prints one JSON line per size and a markdown table at the end; --json also writes the rows to a file.  The paper's own figures (A100-40GB,
-fp32 on CUDA cores, Tables of App. J.1 / K) are printed beside ours as context: another GPU,
-another precision, not a target.
+Prints one JSON line per size and a markdown table at the end; --json also writes the rows to a file.
+The paper's own figures (A100-40GB, fp32 on CUDA cores, Tables of App. J.1 / K) are printed beside ours
+as context: another GPU, another precision, not a target.
 """
 import argparse
 import json
