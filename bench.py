@@ -156,7 +156,7 @@ def run_reference(args, w):
 def fwd_launches(w):
     """Kernels one forward call of the library launches for this workload."""
     if w.mode != wl.MODE_BF16_TC:
-        tiled = w.d <= 64 and w.k <= 32 and (w.N // 128) * w.H >= 296
+        tiled = w.d <= 64 and w.k <= 32 and (w.N // 128) * w.H >= 48
         return 4 if tiled else 3          # plan, sweep, (rescoring), softmax+gather-V
     tc = w.k <= 64 or (w.k <= 128 and w.d <= 64)
     if not tc:

@@ -9,6 +9,13 @@
 
 namespace kmip {
 
+// Groups kept per row by the prefilter sweep for 16 < k <= 32 (k + slack, a multiple of 8); the sweep's pending
+// slots take the shared memory the list leaves.
+#ifndef KMIP_F16_LIST32
+#define KMIP_F16_LIST32 48
+#endif
+constexpr int kF16List32 = KMIP_F16_LIST32;
+
 // Per head: largest squared norm of a query row, of a key row, and of the first 16 elements of a key
 // row (the partial sum after the first tensor-core step of a 32-wide head); float bits, maxima taken
 // with integer atomics (the values are non-negative).

@@ -31,9 +31,19 @@ namespace {
 constexpr int kWarpsPerBlock = 8;
 constexpr unsigned FULL = 0xFFFFFFFFu;
 
-__device__ inline int graph_end_of(const int32_t* offs, int G, int N, int i) {
+// End of the graph that holds node i.  Batches of up to kOffsCached - 1 graphs search a copy of the offsets in
+// shared memory: seven dependent global loads per row would otherwise be the longest chain of a small-graph batch.
+constexpr int kOffsCached = 1024;
+__device__ inline int graph_end_of(const int32_t* offs, const int* s_offs, int G, int N, int i) {
     if (offs == nullptr) return N;
     int a = 0, b = G;
+    if (G < kOffsCached) {
+        while (b - a > 1) {
+            const int m = (a + b) >> 1;
+            if (s_offs[m] <= i) a = m; else b = m;
+        }
+        return max(0, min(N, s_offs[a + 1]));
+    }
     while (b - a > 1) {
         const int m = (a + b) >> 1;
         if (__ldg(offs + m) <= i) a = m; else b = m;
@@ -61,6 +71,11 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
     __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
     __shared__ __align__(16) float s_q[kWarpsPerBlock][D];
     __shared__ uint32_t s_words[kWarpsPerBlock][LIST];
+    __shared__ int s_offs[kOffsCached];
+    if (offs != nullptr && G < kOffsCached) {
+        for (int x = threadIdx.x; x <= G; x += blockDim.x) s_offs[x] = __ldg(offs + x);
+        __syncthreads();
+    }
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     cand_t* row = s_rows[wib];
     float* q = s_q[wib];
@@ -98,7 +113,7 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
 
     for (; r < n_rows; r += stride) {
         const int i = (int)(r / H), h = (int)(r % H);
-        const int hi = graph_end_of(offs, G, N, i);
+        const int hi = graph_end_of(offs, s_offs, G, N, i);
 
         // empty slots: the four-pipeline sweep marks them by the half 0xFFFF and never writes their group word,
         // the ring sweep writes an all-ones word
@@ -264,7 +279,7 @@ cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w) {
     // the list sizes are those of score_select_f16_list
     if (a.k <= 8) { KMIP_LAUNCH_REFINE16(2, 16); }
     else if (a.k <= 16) { KMIP_LAUNCH_REFINE16(2, 24); }
-    else { KMIP_LAUNCH_REFINE16(4, 48); }
+    else { KMIP_LAUNCH_REFINE16(4, kF16List32); }
 #undef KMIP_LAUNCH_REFINE16
     return cudaGetLastError();
 }

@@ -31,6 +31,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "f16_filter.cuh"
 #include "ptx.cuh"
 
 #include <cuda_fp16.h>
@@ -577,13 +578,14 @@ cudaError_t launch_cfg(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
 template <int D, bool DUMP>
 cudaError_t launch_d(const FwdArgs& a, const FwdWorkspace& w, float* dump) {
     // (list blocks, query tiles per CTA, key stages, pending slots per row); shared memory decides
-    return launch_cfg<D, 6, 3, 3, 22, DUMP>(a, w, dump);
+    // the per-warp block of shared memory stays at 14848 bytes: 192 per list slot, 256 per pending slot
+    return launch_cfg<D, kF16List32 / 8, 3, 3, (14848 - kF16List32 * 192) / 256, DUMP>(a, w, dump);
 }
 
 }  // namespace
 
 bool score_select_f16_supported(int32_t d, int32_t k) { return (d == 16 || d == 32) && k <= 32; }
-int score_select_f16_list(int32_t k) { return k <= 8 ? 16 : k <= 16 ? 24 : 48; }
+int score_select_f16_list(int32_t k) { return k <= 8 ? 16 : k <= 16 ? 24 : kF16List32; }
 // lists of up to 24 groups (k <= 16) run the four-pipeline kernel of score_select_f16x4.cu with 512-row work items
 int score_select_f16_rows_per_item(int32_t k) { return k <= 16 ? score_select_f16x4_rows_per_item() : 3 * BM; }
 
