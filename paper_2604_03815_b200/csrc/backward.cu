@@ -37,25 +37,9 @@ bwd_rows_kernel(const T* __restrict__ K, const T* __restrict__ V, const T* __res
         float p[kMaxEntriesPerLane];
         load_row_softmax(topk_idx + (size_t)r * k, topk_score + (size_t)r * k, k, N, scale, lane, j, p);
 
-        // dP_t = g_i . v_{j_t}: each lane owns its entries and walks the d columns
+        // dP_t = g_i . v_{j_t}
         float dP[kMaxEntriesPerLane];
-#pragma unroll
-        for (int e = 0; e < kMaxEntriesPerLane; ++e) dP[e] = 0.0f;
-        const T* g = dOut + (size_t)r * D;
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += VEC) {
-            float gv[VEC];
-            Elem<T>::load_vec(g + c0, gv);
-#pragma unroll
-            for (int e = 0; e < kMaxEntriesPerLane; ++e) {
-                if (e * 32 < k && j[e] >= 0) {
-                    float vv[VEC];
-                    Elem<T>::load_vec(V + ((size_t)j[e] * H + h) * D + c0, vv);
-#pragma unroll
-                    for (int c = 0; c < VEC; ++c) dP[e] = fmaf(gv[c], vv[c], dP[e]);
-                }
-            }
-        }
+        gather_dot<T, D>(V, H, h, k, lane, dOut + (size_t)r * D, j, dP);
         // with dropout the output was sum_t f_t p_t v_t (f constant here): dP_t = f_t (g . v_t), and the
         // weight that reaches dV is f_t p_t
         float f[kMaxEntriesPerLane];

@@ -112,4 +112,42 @@ __device__ __forceinline__ void gather_weighted_sum(const T* __restrict__ X, int
     }
 }
 
+// dots[e] of lane l = g . X[j[e] of lane l, h, :] for the row's entries (entry t in lane t % 32, register t / 32), with
+// the same lane layout as gather_weighted_sum: LPR lanes share one gathered row, one 16-byte load each, so a load
+// instruction touches 32 / LPR rows instead of 32; the partial sums of a row are added across its lanes and handed
+// to the entry's own lane.  g is the row-major vector of D elements at `g_row`.
+template <typename T, int D>
+__device__ __forceinline__ void gather_dot(const T* __restrict__ X, int H, int h, int k, int lane, const T* __restrict__ g_row,
+                                           const int (&j)[kMaxEntriesPerLane], float (&dots)[kMaxEntriesPerLane]) {
+    constexpr int VEC = Elem<T>::kVec;
+    constexpr int LPR = D / VEC;
+    constexpr int EPW = 32 / LPR;
+    const int part = lane % LPR, sub = lane / LPR;
+    float gv[VEC];
+    Elem<T>::load_vec(g_row + part * VEC, gv);
+#pragma unroll
+    for (int e = 0; e < kMaxEntriesPerLane; ++e) {
+        dots[e] = 0.0f;
+        if (e * 32 < k) {
+#pragma unroll
+            for (int base = 0; base < 32; base += EPW) {
+                if (e * 32 + base >= k) break;
+                const int jj = __shfl_sync(0xFFFFFFFFu, j[e], base + sub);
+                float s = 0.0f;
+                if (jj >= 0) {
+                    float v[VEC];
+                    Elem<T>::load_vec(X + ((size_t)jj * H + h) * D + part * VEC, v);
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) s = fmaf(gv[c], v[c], s);
+                }
+#pragma unroll
+                for (int o = 1; o < LPR; o <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+                // the entry of lane l was gathered by the lanes (l % EPW) * LPR ... in the round base = l - l % EPW
+                const float t = __shfl_sync(0xFFFFFFFFu, s, (lane % EPW) * LPR);
+                if (lane - lane % EPW == base) dots[e] = t;
+            }
+        }
+    }
+}
+
 }  // namespace kmip

@@ -63,3 +63,27 @@ def test_static_scratch_forward_matches_regular_forward_twice(mode):
     torch.cuda.synchronize()
     assert rc == kb.KMIP_OK and int(status.item()) == kb.KMIP_OK
     pu.check_forward(first, got)
+
+
+@pytest.mark.gpu
+def test_static_scratch_empty_batch_and_no_status_pointer():
+    """N = 0 enqueues no kernel but must clear a status word the caller polls (it may hold the previous
+    call's error); device_status = NULL is allowed on every path."""
+    from paper_2604_03815_b200 import binding as kb
+    from tests import parity_util as pu
+    w = wl.iid_workload("a", 902, [300, 40], 2, 16, 8, wl.MODE_BF16_TC)
+    Q, K, V, dO, offs = pu.to_device(w)
+    got = kb.ForwardBuffers(w.N, w.G, w.H, w.d, w.k, w.mode)
+    status = torch.full((1,), kb.KMIP_ERR_BAD_OFFSETS, dtype=torch.int32, device="cuda")   # a stale error
+    e = torch.empty((0, w.H, w.d), dtype=Q.dtype, device="cuda")
+    ei, es = torch.empty((0, w.H, w.k), dtype=torch.int32, device="cuda"), torch.empty((0, w.H, w.k), device="cuda")
+    rc = kb.kmip_attn_forward_static_scratch(e, e, e, None, w.k, w.mode, e, ei, es, device_status=status)
+    torch.cuda.synchronize()
+    assert rc == kb.KMIP_OK and int(status.item()) == kb.KMIP_OK
+    rc = kb.kmip_attn_forward_static_scratch(e, e, e, None, w.k, w.mode, e, ei, es, device_status=None)
+    assert rc == kb.KMIP_OK
+    rc = kb.kmip_attn_forward_static_scratch(Q, K, V, offs, w.k, w.mode, got.out, got.topk_idx, got.topk_score,
+                                             device_status=None)
+    torch.cuda.synchronize()
+    assert rc == kb.KMIP_OK
+    pu.check_forward(w, got)
