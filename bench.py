@@ -427,11 +427,13 @@ def run_ours(args, w):
                "so this is a cache-warm figure (the headline workload is config 4)")
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True,
+        "scaling": "strong" if getattr(args, "sharded", False) else "weak", "vs_baseline": None,
         "dtype": "bf16" if w.mode == wl.MODE_BF16_TC else "f32", "data": "synthetic",
         "config": {"workload": describe(w), "passes": "forward+backward" if w.backward else "forward",
                    "l2": l2_note,
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": ("whole graphs per rank, no exchange" if getattr(args, "sharded", False)
+                                   else "replicas only" if world > 1 else "single GPU")},
         "roofline": roofline,
         "stages_ms": {k_: round(v, 4) for k_, v in per_call.items()},
         "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
@@ -479,6 +481,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pruned", action="store_true", help="skip the extra measurement of the pruned mode")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the short runs of configs 3 and 5")
+    ap.add_argument("--shard", choices=["replicas", "graphs"], default="replicas",
+                    help="N > 1: independent replicas (default, weak scaling) or the batch's graphs split over the "
+                         "ranks (strong scaling; needs at least as many graphs as ranks, e.g. --config 5 on 2 or 4 GPUs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -487,6 +492,15 @@ def main():
         return
     kw = {"N": args.nodes} if args.nodes and args.config in (3, 4) else {}
     w = wl.make_config(args.config, **kw)
+    args.sharded = args.shard == "graphs" and world > 1 and args.impl == "ours" and w.G >= world
+    if args.sharded:
+        # this rank's contiguous run of graphs; a query only sees its own graph, so nothing is exchanged
+        import dataclasses
+        import numpy as np
+        lo, hi, offs, _ = kdist.shard_of(w.graph_offsets, world, rank)
+        w = dataclasses.replace(w, graph_offsets=np.asarray(offs, dtype=np.int32), Q=w.Q[lo:hi], K=w.K[lo:hi],
+                                V=w.V[lo:hi], dOut=w.dOut[lo:hi])
+        args.no_pruned = args.no_other_configs = True
     res = run_reference(args, w) if args.impl == "reference" else run_ours(args, w)
     if res is not None:
         print(json.dumps(res), flush=True)
