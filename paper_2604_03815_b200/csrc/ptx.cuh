@@ -314,6 +314,21 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// s + a.lo * b.lo, then + a.hi * b.hi, with a and b pairs of bf16 values and s fp32: the product of two bf16 values
+// is exact in fp32, so each step is bit for bit fmaf(float(a), float(b), s) without the two conversions (sm_100+).
+__device__ __forceinline__ float fma_bf16_pair(uint32_t a, uint32_t b, float s) {
+    asm("{\n\t"
+        ".reg .b16 al, ah, bl, bh;\n\t"
+        "mov.b32 {al, ah}, %1;\n\t"
+        "mov.b32 {bl, bh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, al, bl, %0;\n\t"
+        "fma.rn.f32.bf16 %0, ah, bh, %0;\n\t"
+        "}"
+        : "+f"(s)
+        : "r"(a), "r"(b));
+    return s;
+}
+
 // 16-byte asynchronous copy global -> shared that bypasses L1 (both addresses 16-byte aligned); copies issued by a
 // thread complete in groups: commit closes a group, wait<N> returns when all but the newest N groups have landed
 __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {

@@ -7,7 +7,8 @@
 //      whose maximum g satisfies g + err(g) < lowS cannot hold one of the k best keys: it is skipped.
 //      err(T) = a + r |T| bounds |fp16 score - exact scaled score| (f16_filter.cuh).
 //   2. The keys of the other groups are scored again - fp32 fused multiply-adds over the bf16 values in
-//      index order, read from K in place - and the k best under (score desc, key asc) are kept with the
+//      index order (the mixed-precision instruction: exact product, one rounding, the same bits as convert +
+//      fmaf), read from K in place - and the k best under (score desc, key asc) are kept with the
 //      running top-k buffer of the CUDA-core kernel.
 //   3. If the sweep's list was full, groups it dropped have maxima at most g_min, the smallest one
 //      kept.  When g_min + err(g_min) reaches the k-th best exact score found, a dropped group could
@@ -69,7 +70,7 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
     constexpr int KSTEPS = D / 16;
     static_assert(E <= 4 && LIST <= 64 && D <= 32, "k <= 32, head widths 16 and 32");
     __shared__ cand_t s_rows[kWarpsPerBlock][CAP];
-    __shared__ __align__(16) float s_q[kWarpsPerBlock][D];
+    __shared__ __align__(16) unsigned short s_qb[kWarpsPerBlock][D];  // the query row, bf16 bits
     __shared__ uint32_t s_words[kWarpsPerBlock][LIST];
     __shared__ int s_offs[kOffsCached];
     if (offs != nullptr && G < kOffsCached) {
@@ -78,7 +79,6 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
     }
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     cand_t* row = s_rows[wib];
-    float* q = s_q[wib];
     uint32_t* words = s_words[wib];
     const long long n_rows = (long long)N * H;
     const long long stride = (long long)gridDim.x * kWarpsPerBlock;
@@ -131,7 +131,7 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
         }
         const float qc = nx_q;
         __syncwarp();
-        if (lane < D) q[lane] = qc;
+        if (lane < D) s_qb[wib][lane] = (unsigned short)(__float_as_uint(qc) >> 16);  // exact: the value came from bf16
         for (int t = lane; t < k; t += 32) row[t] = 0ull;
         fetch(r + stride);
 
@@ -209,6 +209,13 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
             }
             ptx::cp_async_commit();  // an empty group when there is nothing left, so that the count below holds
         };
+        uint32_t qp[D / 2];  // the query row, two bf16 values to a register
+        __syncwarp();
+#pragma unroll
+        for (int v = 0; v < D / 8; ++v) {
+            const uint4 t4 = *reinterpret_cast<const uint4*>(&s_qb[wib][v * 8]);
+            qp[v * 4 + 0] = t4.x; qp[v * 4 + 1] = t4.y; qp[v * 4 + 2] = t4.z; qp[v * 4 + 3] = t4.w;
+        }
         issue(0);
         for (int step = 0; step < nsteps; ++step) {
             issue(step + 1);
@@ -225,13 +232,8 @@ refine_f16_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __re
                 for (int v = 0; v < P; ++v) {
                     const uint4 rw = *reinterpret_cast<const uint4*>(kr + v * 16);
                     const uint32_t wv[4] = {rw.x, rw.y, rw.z, rw.w};
-                    const float4 qa = *reinterpret_cast<const float4*>(q + v * 8), qb = *reinterpret_cast<const float4*>(q + v * 8 + 4);
-                    const float qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        s = fmaf(qv[2 * x], __uint_as_float(wv[x] << 16), s);
-                        s = fmaf(qv[2 * x + 1], __uint_as_float(wv[x] & 0xFFFF0000u), s);
-                    }
+                    for (int x = 0; x < 4; ++x) s = ptx::fma_bf16_pair(qp[v * 4 + x], wv[x], s);
                 }
             }
             const bool pass = kv && (s > tau);
